@@ -1,0 +1,196 @@
+/*
+ * dscale.h -- C ABI of the DScale verify-side hot path for NVIDIA B200 (sm_100a).
+ *
+ * One decode step of block-diffusion speculative decoding verifies, for each
+ * of N live requests, a window of W = 16 slots (slot 0 = the known anchor,
+ * slots 1..15 = draft candidates).  This library implements the three
+ * verify-side stages of that step:
+ *
+ *   dscale_alloc_verify   DVL allocation and flat-pack   (Algorithm 1, Eq. 6-11)
+ *   dscale_verify_attn    packed ragged verify attention (Section 3.2, Eq. 2, Eq. 15)
+ *   dscale_accept         greedy prefix verification     ("Prefix verifier", Algorithm 2)
+ *
+ * General rules
+ * -------------
+ *  - Unless a parameter is marked HOST, every pointer is a DEVICE pointer that
+ *    the caller owns; the library never allocates, frees or synchronises.
+ *  - Every call only enqueues kernels on `stream` (a cudaStream_t passed as
+ *    void*).  All shapes are fixed by the arguments, every data-dependent
+ *    quantity (N, lengths, offsets, context lengths) is read on the device,
+ *    and all intermediate state lives at fixed addresses inside the caller's
+ *    workspace (Eq. 12): a CUDA graph captured once over these calls can be
+ *    replayed with new inputs written to the same addresses.
+ *  - Return value: DSCALE_OK, or a negative DSCALE_ERR_* code, in which case
+ *    nothing was enqueued.  Faults that only the device can see (a page id out
+ *    of range, a NaN score, a bounded wait that ran out) are reported through
+ *    the sticky status word in the workspace (dscale_ws_field(.., DSCALE_WS_STATUS));
+ *    the kernels stay in bounds in that case and finish.
+ *  - Fixed by this build: W = 16, head_dim = 128, KV page = 16 tokens,
+ *    budget = 8 slots per live request, n_bs <= DSCALE_MAX_NBS.
+ *
+ * Layouts
+ * -------
+ *  KV cache (one layer):  bf16 [num_pages][n_kv_heads][16][128]; logical token t
+ *      of request i lives in page block_table[i][t / 16], slot t % 16.
+ *  Packed rows:           row s = offset_i + j holds slot j of request i
+ *      (Eq. 11); M_bs = 8 * n_bs rows are always present, M_live = 8 * N are live.
+ *  q / out:               bf16 [M_bs][n_q_heads][128]; q-head h uses kv-head
+ *      h / (n_q_heads / n_kv_heads).
+ *  logits:                fp32 [M_bs][ld], ld >= vocab, ld % 4 == 0.
+ */
+#ifndef DSCALE_H_
+#define DSCALE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DSCALE_W 16
+#define DSCALE_HEAD_DIM 128
+#define DSCALE_PAGE 16
+#define DSCALE_MAX_NBS 64
+
+enum {
+  DSCALE_OK = 0,
+  DSCALE_ERR_INVALID_ARG = -1,   /* null / misaligned pointer, size out of range  */
+  DSCALE_ERR_UNSUPPORTED = -2,   /* shape this build has no kernel for            */
+  DSCALE_ERR_CUDA = -3,          /* a CUDA runtime / driver call failed           */
+  DSCALE_ERR_WORKSPACE = -4      /* workspace too small or not initialised        */
+};
+
+/* bits of the device status word (0 = OK; bits are OR-ed, sticky until
+ * dscale_workspace_init is called again) */
+enum {
+  DSCALE_STATUS_OK = 0,
+  DSCALE_STATUS_BAD_SCORE = 1,   /* score NaN or outside [0,1] (clamped)          */
+  DSCALE_STATUS_BAD_PAGE = 2,    /* page id outside [0, num_pages) (page 0 used)  */
+  DSCALE_STATUS_BAD_LEN = 4,     /* N or a context length out of range (clamped)  */
+  DSCALE_STATUS_TIMEOUT = 8      /* a bounded device-side wait ran out            */
+};
+
+/* fields readable through dscale_ws_field */
+enum {
+  DSCALE_WS_STATUS = 0,     /* int32 [1]                                              */
+  DSCALE_WS_K = 1,          /* int32 [n_bs]      verify lengths k_i (0 for sentinels) */
+  DSCALE_WS_OFFSET = 2,     /* int32 [n_bs + 1]  Eq. 10, sentinels = M_live           */
+  DSCALE_WS_Q_START = 3,    /* int32 [n_bs]      offset_i            (Alg. 2 l.14-16) */
+  DSCALE_WS_Q_END = 4,      /* int32 [n_bs]      offset_i + k_i                       */
+  DSCALE_WS_TOKENS = 5,     /* int32 [8 n_bs]    packed token ids                     */
+  DSCALE_WS_POSITIONS = 6,  /* int32 [8 n_bs]    packed positions ctx_i + j           */
+  DSCALE_WS_KV_REFS = 7,    /* int32 [8 n_bs]    packed cache slots page*16 + t%16    */
+  DSCALE_WS_ROW_REQ = 8,    /* int32 [8 n_bs]    request of each packed row, -1 tail  */
+  DSCALE_WS_TOP1 = 9,       /* int32 [8 n_bs]    target argmax per packed row         */
+  DSCALE_WS_K0 = 10,        /* int32 [n_bs]      seed lengths of Eq. 7                */
+  DSCALE_WS_N_LIVE = 11     /* int32 [1]         N as seen by the last allocation     */
+};
+
+/*
+ * Size in bytes of the workspace for capacity n_bs (the paper's N_bs) and the
+ * given head geometry.  num_sms = number of SMs of the device the calls will
+ * run on (it fixes the persistent attention grid and its split-KV scratch).
+ * Returns 0 for unsupported arguments.  HOST call, no CUDA activity.
+ */
+size_t dscale_workspace_bytes(int n_bs, int n_q_heads, int n_kv_heads, int head_dim, int num_sms);
+
+/*
+ * Prepare a workspace: zeroes the status word, the counters and the index
+ * sections (the Alloc(N_bs, 8 N_bs) of Algorithm 2, line 4).  ws must be
+ * 256-byte aligned device memory of at least dscale_workspace_bytes(...).
+ * Call once, before capturing or running the other calls.
+ */
+int dscale_workspace_init(void* ws, size_t bytes, int n_bs, int n_q_heads, int n_kv_heads,
+                          int head_dim, int num_sms, void* stream);
+
+/*
+ * DVL allocation and flat-pack (Algorithm 1 from its second line; Eq. 6, 7, 9, 10, 11).
+ *
+ *   n_live        [1]  N, 1 <= N <= n_bs, read on the device
+ *   scores        fp32 [n_bs][15]; slot j = 1..15.  scores_are_logits = 0: the
+ *                 values are per-position acceptance probabilities in [0,1];
+ *                 = 1: predictor logits, the sigmoid of Algorithm 1 is applied.
+ *                 A running minimum (Eq. 6) is always applied.
+ *   draft_tokens  int32 [n_bs][16]; slot 0 = anchor
+ *   ctx_len       int32 [n_bs]; tokens of request i already in the cache, the
+ *                 anchor excluded.  The K/V of slot j is expected at logical
+ *                 position ctx_len[i] + j.
+ *   block_table   int32 [n_bs][max_pages]
+ *
+ * Writes into the workspace: Q, k0, k, offset, q_start, q_end, packed tokens,
+ * positions (ctx_i + j), kv_refs (page * 16 + slot), row_req, the sentinels of
+ * Algorithm 1's last two lines, and the tile schedule the attention kernel
+ * reads.  sum_i k_i = 8 N exactly, 1 <= k_i <= 16, ties in the grow / shrink
+ * choice go to the lowest request index.  One kernel, one thread block.
+ */
+int dscale_alloc_verify(void* ws, int n_bs, const int32_t* n_live, const float* scores,
+                        int scores_are_logits, const int32_t* draft_tokens,
+                        const int32_t* ctx_len, const int32_t* block_table, int max_pages,
+                        int num_pages, void* stream);
+
+/*
+ * Packed ragged verify attention for one layer (Section 3.2; Eq. 15 and the
+ * sentence after it).  For live request i, row j < k_i, q-head h:
+ *     out[offset_i + j][h] = softmax(q[offset_i + j][h] . K^T * sm_scale) V
+ * over the logical keys 0 .. positions[offset_i + j] of request i (its whole
+ * committed context and the window slots up to j), kv-head h / group.  Rows
+ * at or beyond M_live are written as zero.  Lengths, offsets and positions are
+ * the ones dscale_alloc_verify left in the workspace.
+ *
+ * The query tile is sized to the live rows: one 64-row tensor-core tile holds
+ * the 4 q-heads of a GQA group times the <= 16 window rows, so each K/V page is
+ * read from HBM once per kv-head.  Requires n_q_heads / n_kv_heads == 4;
+ * returns DSCALE_ERR_UNSUPPORTED otherwise (use dscale_verify_attn_simt).
+ *
+ *   q, out        bf16 [8 n_bs][n_q_heads][128], 16-byte aligned
+ *   k_cache, v_cache  bf16 [num_pages][n_kv_heads][16][128], 16-byte aligned
+ */
+int dscale_verify_attn(void* ws, int n_bs, const void* q, const void* k_cache,
+                       const void* v_cache, const int32_t* block_table, int max_pages,
+                       int num_pages, int n_q_heads, int n_kv_heads, float sm_scale, void* out,
+                       void* stream);
+
+/*
+ * Same operation and arguments on plain CUDA cores (no tensor cores, any GQA
+ * group size that divides n_q_heads).  Slow; kept as the in-library
+ * cross-check of the tensor-core kernel and for shapes it does not cover.
+ */
+int dscale_verify_attn_simt(void* ws, int n_bs, const void* q, const void* k_cache,
+                            const void* v_cache, const int32_t* block_table, int max_pages,
+                            int num_pages, int n_q_heads, int n_kv_heads, float sm_scale,
+                            void* out, void* stream);
+
+/*
+ * Greedy prefix verification and output building ("Prefix verifier" paragraph;
+ * Algorithm 2, lines 21-26).  top1[s] = first index of the maximum of
+ * logits[s][0..vocab) for s < M_live (a NaN never counts as a maximum).
+ * Request i accepts candidates while top1[offset_i + a] == tokens[offset_i + a + 1],
+ * a < k_i - 1; the successor is top1[offset_i + a_i].
+ *
+ *   accept_len   int32 [n_bs]      a_i (0 for sentinels)
+ *   next_anchor  int32 [n_bs]      successor token (-1 for sentinels)
+ *   out_tokens   int32 [n_bs][16]  accepted candidates, then the successor, then -1
+ *   out_len      int32 [n_bs]      a_i + 1 (0 for sentinels)
+ *   ctx_len_inout  nullable; if given, ctx_len[i] += a_i + 1 for live i (the
+ *                 boundary write-back; not idempotent across replays)
+ */
+int dscale_accept(void* ws, int n_bs, const float* logits, int64_t ld, int vocab,
+                  int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
+                  int32_t* out_len, int32_t* ctx_len_inout, void* stream);
+
+/*
+ * Device address of a workspace field (see DSCALE_WS_*), for tests and for
+ * callers that feed packed fields to other kernels.  HOST call; returns NULL
+ * for a bad field id.  The address depends only on (ws, n_bs).
+ */
+const int32_t* dscale_ws_field(const void* ws, int n_bs, int field);
+
+/* Number of kernels the three stage calls enqueue (for launch accounting):
+ * which = 0 alloc, 1 attention, 2 accept, 3 attention (simt). */
+int dscale_launches_per_call(int which);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* DSCALE_H_ */

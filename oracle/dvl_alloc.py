@@ -159,7 +159,9 @@ def dvl_alloc(n_bs: int, n_live: int, scores, draft_tokens, ctx_len, block_table
         positions[s] = 0
         kv_refs[s] = tail_ref
 
-    return dict(k=k, k0=np.asarray(k0, dtype=np.int32), offset=offset,
+    k0_full = np.zeros(n_bs, dtype=np.int32)
+    k0_full[:N] = k0
+    return dict(k=k, k0=k0_full, offset=offset,
                 q_start=offset[:-1].copy(), q_end=(offset[:-1] + k).astype(np.int32),
                 tokens=tokens, positions=positions, kv_refs=kv_refs, row_req=row_req,
                 Q=Q, n_updates=n_updates, m_live=M_live)

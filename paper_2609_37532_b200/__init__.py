@@ -1,0 +1,12 @@
+"""B200-native DScale verify path: thin Python binding over libdscale.so.
+
+Every step of the path runs in the CUDA library; this package only marshals
+torch tensors (device memory, streams) into the C ABI declared in
+include/dscale.h.  There is no CPU fallback: importing the binding without the
+built library raises.
+"""
+from .binding import (DScaleError, VerifyWorkspace, accept, alloc_verify, lib, verify_attn,
+                      verify_attn_simt, WS_FIELDS)
+
+__all__ = ["DScaleError", "VerifyWorkspace", "accept", "alloc_verify", "lib", "verify_attn",
+           "verify_attn_simt", "WS_FIELDS"]

@@ -1,0 +1,142 @@
+"""ctypes binding of include/dscale.h.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libdscale.so")
+
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2609_37532_b200.build` "
+        "(there is no fallback path)")
+
+lib = C.CDLL(_LIB_PATH)
+
+_vp, _i, _i64, _f, _sz = C.c_void_p, C.c_int, C.c_int64, C.c_float, C.c_size_t
+lib.dscale_workspace_bytes.restype = _sz
+lib.dscale_workspace_bytes.argtypes = [_i, _i, _i, _i, _i]
+lib.dscale_workspace_init.restype = _i
+lib.dscale_workspace_init.argtypes = [_vp, _sz, _i, _i, _i, _i, _i, _vp]
+lib.dscale_alloc_verify.restype = _i
+lib.dscale_alloc_verify.argtypes = [_vp, _i, _vp, _vp, _i, _vp, _vp, _vp, _i, _i, _vp]
+for _name in ("dscale_verify_attn", "dscale_verify_attn_simt"):
+    getattr(lib, _name).restype = _i
+    getattr(lib, _name).argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _f, _vp, _vp]
+lib.dscale_accept.restype = _i
+lib.dscale_accept.argtypes = [_vp, _i, _vp, _i64, _i, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.dscale_ws_field.restype = _vp
+lib.dscale_ws_field.argtypes = [_vp, _i, _i]
+lib.dscale_launches_per_call.restype = _i
+lib.dscale_launches_per_call.argtypes = [_i]
+
+WS_FIELDS = dict(status=0, k=1, offset=2, q_start=3, q_end=4, tokens=5, positions=6, kv_refs=7,
+                 row_req=8, top1=9, k0=10, n_live=11)
+_ERR = {-1: "invalid argument", -2: "unsupported shape", -3: "CUDA error", -4: "workspace"}
+
+
+class DScaleError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where}: {_ERR.get(code, 'error')} ({code})")
+        self.code = code
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise DScaleError(rc, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _need(t: torch.Tensor, dtype, name: str):
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+
+
+class VerifyWorkspace:
+    """The fixed-address workspace of one captured capacity n_bs."""
+
+    def __init__(self, n_bs: int, n_q_heads: int, n_kv_heads: int, head_dim: int = 128,
+                 device=None):
+        device = torch.device("cuda" if device is None else device)
+        self.n_bs, self.n_q_heads, self.n_kv_heads, self.head_dim = n_bs, n_q_heads, n_kv_heads, head_dim
+        self.num_sms = torch.cuda.get_device_properties(device).multi_processor_count
+        nbytes = lib.dscale_workspace_bytes(n_bs, n_q_heads, n_kv_heads, head_dim, self.num_sms)
+        if nbytes == 0:
+            raise DScaleError(-2, "dscale_workspace_bytes")
+        self.nbytes = nbytes
+        self.buf = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+        off = (-self.buf.data_ptr()) % 256
+        self.ptr = self.buf.data_ptr() + off
+        with torch.cuda.device(device):
+            _check(lib.dscale_workspace_init(C.c_void_p(self.ptr), nbytes, n_bs, n_q_heads,
+                                             n_kv_heads, head_dim, self.num_sms, _stream()),
+                   "dscale_workspace_init")
+
+    def field(self, name: str) -> torch.Tensor:
+        """int32 view of a workspace section (shares memory with the workspace)."""
+        n_bs = self.n_bs
+        sizes = dict(status=1, n_live=1, k=n_bs, k0=n_bs, offset=n_bs + 1, q_start=n_bs,
+                     q_end=n_bs, tokens=8 * n_bs, positions=8 * n_bs, kv_refs=8 * n_bs,
+                     row_req=8 * n_bs, top1=8 * n_bs)
+        addr = lib.dscale_ws_field(C.c_void_p(self.ptr), n_bs, WS_FIELDS[name])
+        start = (addr - self.buf.data_ptr())
+        return self.buf[start:start + 4 * sizes[name]].view(torch.int32)
+
+    def status(self) -> int:
+        return int(self.field("status").item())
+
+
+def alloc_verify(ws: VerifyWorkspace, n_live, scores, draft_tokens, ctx_len, block_table,
+                 num_pages: int, scores_are_logits: bool = False):
+    _need(n_live, torch.int32, "n_live"); _need(scores, torch.float32, "scores")
+    _need(draft_tokens, torch.int32, "draft_tokens"); _need(ctx_len, torch.int32, "ctx_len")
+    _need(block_table, torch.int32, "block_table")
+    assert scores.shape == (ws.n_bs, 15) and draft_tokens.shape == (ws.n_bs, 16)
+    assert ctx_len.shape == (ws.n_bs,) and block_table.shape[0] == ws.n_bs
+    _check(lib.dscale_alloc_verify(C.c_void_p(ws.ptr), ws.n_bs, _ptr(n_live), _ptr(scores),
+                                   int(scores_are_logits), _ptr(draft_tokens), _ptr(ctx_len),
+                                   _ptr(block_table), block_table.shape[1], num_pages, _stream()),
+           "dscale_alloc_verify")
+
+
+def _attn(fn, name, ws, q, k_cache, v_cache, block_table, sm_scale, out):
+    _need(q, torch.bfloat16, "q"); _need(k_cache, torch.bfloat16, "k_cache")
+    _need(v_cache, torch.bfloat16, "v_cache"); _need(out, torch.bfloat16, "out")
+    _need(block_table, torch.int32, "block_table")
+    assert q.shape == (8 * ws.n_bs, ws.n_q_heads, 128) and out.shape == q.shape
+    assert k_cache.shape[1:] == (ws.n_kv_heads, 16, 128) and v_cache.shape == k_cache.shape
+    _check(fn(C.c_void_p(ws.ptr), ws.n_bs, _ptr(q), _ptr(k_cache), _ptr(v_cache),
+              _ptr(block_table), block_table.shape[1], k_cache.shape[0], ws.n_q_heads,
+              ws.n_kv_heads, float(sm_scale), _ptr(out), _stream()), name)
+
+
+def verify_attn(ws, q, k_cache, v_cache, block_table, sm_scale, out):
+    _attn(lib.dscale_verify_attn, "dscale_verify_attn", ws, q, k_cache, v_cache, block_table,
+          sm_scale, out)
+
+
+def verify_attn_simt(ws, q, k_cache, v_cache, block_table, sm_scale, out):
+    _attn(lib.dscale_verify_attn_simt, "dscale_verify_attn_simt", ws, q, k_cache, v_cache,
+          block_table, sm_scale, out)
+
+
+def accept(ws, logits, vocab: int, accept_len, next_anchor, out_tokens, out_len,
+           ctx_len_inout=None):
+    _need(logits, torch.float32, "logits")
+    for n, t in (("accept_len", accept_len), ("next_anchor", next_anchor),
+                 ("out_tokens", out_tokens), ("out_len", out_len)):
+        _need(t, torch.int32, n)
+    assert logits.shape[0] == 8 * ws.n_bs and out_tokens.shape == (ws.n_bs, 16)
+    _check(lib.dscale_accept(C.c_void_p(ws.ptr), ws.n_bs, _ptr(logits), logits.stride(0), vocab,
+                             _ptr(accept_len), _ptr(next_anchor), _ptr(out_tokens), _ptr(out_len),
+                             _ptr(ctx_len_inout), _stream()), "dscale_accept")

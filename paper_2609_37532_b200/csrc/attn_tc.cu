@@ -1,0 +1,713 @@
+// Packed ragged verify attention on the sm_100a tensor cores.
+//
+// Shape of the work.  Per live request i and kv-head g the query tile is the
+// GQA group's 4 q-heads x the k_i <= 16 live window rows = at most 64 rows:
+// exactly one M = 64 tcgen05 tile (row m = 4 j + h_local), instead of the
+// 128-row prefill tile that would leave 112 masked rows per request and head
+// (Eq. 2).  Keys and values are streamed once per kv-head in tiles of 128
+// tokens (8 pages).  The kernel is HBM-bound; the tensor cores only have to
+// keep up with the K/V stream.
+//
+// Schedule.  The key tiles of all (request, kv-head) pairs form one linear
+// list (the per-request tile prefix comes from the allocation kernel); CTA c
+// of a persistent grid of one CTA per SM takes the contiguous slice
+// [c T / C, (c+1) T / C).  A slice cuts at most its first and its last pair;
+// those write an un-normalised partial (O, m, l) to the workspace, and the
+// last CTA to arrive at a pair (a ticket counter, nobody waits) merges the
+// partials and writes the rows.  Pairs inside a slice are written directly.
+// The grid and every address are independent of the lengths, so a captured
+// launch replays at any mix of lengths.
+//
+// Pipeline inside a CTA (192 threads):
+//   warp 4     producer: per tile, 16 + 16 TMA box copies (one 16-token page
+//              x 64 columns each, 128-byte swizzle) of K then V into a 5-deep
+//              ring of 32 KB slots; page ids are fetched one tile ahead.
+//   warp 5     one thread issues tcgen05.mma: S = Q K^T (M64 N128 K128, bf16 in,
+//              fp32 in TMEM) for tile t, then O_t = P_{t-1} V_{t-1}; completion
+//              is signalled with tcgen05.commit on mbarriers.
+//   warps 0-3  softmax: thread (w, l < 16) owns row 16 w + l (TMEM lane 32 w + l),
+//              reads S with tcgen05.ld, keeps the running max / sum, writes P as
+//              bf16 into swizzled shared memory for the second MMA, and folds
+//              each per-tile product O_t (read back from TMEM) into fp32
+//              accumulators in registers, rescaled by exp2(m_old - m_new).
+// S and O_t are double-buffered in TMEM (4 x 128 columns), P and Q in shared
+// memory, so the MMA of tile t+1 overlaps the softmax of tile t.
+//
+// Every wait is bounded: when a wait runs out the CTA sets the TIMEOUT status
+// bit, stops issuing work, drains its outstanding copies and releases TMEM.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <map>
+#include <mutex>
+
+#include "kernels.cuh"
+
+namespace dscale {
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kSoftmaxThreads = 128;
+constexpr int kStages = 5;
+constexpr int kSlotBytes = kTileTok * kD * 2;           // 32 KB: one K or V tile
+constexpr int kHalfSlot = kSlotBytes / 2;               // one 64-column half [128 tok][128 B]
+constexpr int kQBytes = kTcRows * kD * 2;               // 16 KB
+constexpr int kPBytes = kTcRows * kTileTok * 2;         // 16 KB
+constexpr int kPageBoxBytes = kPage * 64 * 2;           // 2 KB per TMA box
+constexpr long long kWaitCycles = 1LL << 31;            // ~1 s bound on every wait
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr int kOffQ = 0;                                 // 2 x 16 KB
+constexpr int kOffP = kOffQ + 2 * kQBytes;               // 2 x 16 KB
+constexpr int kOffKV = kOffP + 2 * kPBytes;              // 5 x 32 KB
+constexpr int kOffBar = kOffKV + kStages * kSlotBytes;   // mbarriers
+constexpr int kNumBars = 2 * kStages + 2 + 2 + 2 + 2 + 2 + 1;
+constexpr int kOffMisc = kOffBar + 8 * 24;               // tmem base, abort flag, ticket
+constexpr int kOffTile = kOffMisc + 32;                  // tile prefix, kMaxNbs + 1 ints
+constexpr int kSmemUse = kOffTile + (kMaxNbs + 1) * 4 + 12;
+constexpr int kSmemBytes = kSmemUse + 1024;              // slack for base alignment
+static_assert(kNumBars <= 24, "barrier area");
+static_assert(kSmemBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
+
+enum Bar { B_KV_FULL = 0, B_KV_EMPTY = kStages, B_Q_FULL = 2 * kStages, B_Q_EMPTY = B_Q_FULL + 2,
+           B_S_FULL = B_Q_EMPTY + 2, B_P_FULL = B_S_FULL + 2, B_O_FULL = B_P_FULL + 2,
+           B_GROUP = B_O_FULL + 2 };
+
+// ------------------------------------------------------------------ PTX glue
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the time limit passed or another role of
+// this CTA already gave up (abort flag in shared memory).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+  }
+}
+__device__ __forceinline__ void fence_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+// shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// instruction descriptor: bf16 x bf16 -> fp32, M = 64, N = 128; B is K-major
+// for S = Q K^T and MN-major (tokens are the K dimension) for O = P V
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) |
+                                ((64u >> 4) << 24);
+constexpr uint32_t kIdescS = kIdescBase;
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);
+
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                     uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c,
+                                             uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c),
+               "r"(d) : "memory");
+}
+
+// ------------------------------------------------------------------ schedule
+// One maximal run of tiles of a single (request, kv-head) pair inside a CTA's slice.
+struct Segment {
+  int i, g;          // request, kv-head
+  int t0, t1;        // tile range of the pair covered here
+  int n_tiles;       // tiles of the whole pair
+  bool first_of_cta; // the run starts at the slice start
+};
+
+struct Scheduler {
+  const int* tile_pre;   // shared copy, [n_bs + 1]
+  int n_bs, n_kv;
+  long long pos, end, begin;
+  int i;                 // search hint
+
+  __device__ void init(const int* tp, int n_bs_, int n_kv_, long long b, long long e) {
+    tile_pre = tp; n_bs = n_bs_; n_kv = n_kv_; begin = pos = b; end = e; i = 0;
+  }
+  __device__ bool next(Segment& s) {
+    if (pos >= end) return false;
+    while (i < n_bs && (long long)tile_pre[i + 1] * n_kv <= pos) ++i;
+    const int n_i = tile_pre[i + 1] - tile_pre[i];
+    const long long rem = pos - (long long)tile_pre[i] * n_kv;
+    s.i = i;
+    s.g = (int)(rem / n_i);
+    s.t0 = (int)(rem % n_i);
+    const long long room = end - pos;
+    s.t1 = (int)((long long)(n_i - s.t0) <= room ? n_i : s.t0 + room);
+    s.n_tiles = n_i;
+    s.first_of_cta = (pos == begin);
+    pos += s.t1 - s.t0;
+    return true;
+  }
+};
+
+__device__ __forceinline__ long long slice_begin(int c, long long T, int C) { return (long long)c * T / C; }
+// the CTA whose slice holds linear tile index L
+__device__ __forceinline__ int cta_of(long long L, long long T, int C) {
+  return (int)(((L + 1) * C + T - 1) / T) - 1;
+}
+
+// --------------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
+               const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v) {
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t raw = smem_u32(smem_dyn);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* sm = smem_dyn + (base - raw);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm + kOffMisc);
+  int* s_ticket = reinterpret_cast<int*>(sm + kOffMisc + 8);
+  volatile int* s_dummy = reinterpret_cast<volatile int*>(sm + kOffMisc + 12);
+  int* s_tile = reinterpret_cast<int*>(sm + kOffTile);
+  auto bar = [&](int b) { return base + kOffBar + 8u * b; };
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int c = blockIdx.x;
+  int* hdr = ws_ptr<int>(a.ws, L.hdr);
+  const int n_bs = a.n_bs, n_kv = a.n_kv_heads, Hq = a.n_q_heads;
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(bar(B_KV_FULL + s), 1); mbar_init(bar(B_KV_EMPTY + s), 1); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar(B_Q_FULL + b), 1); mbar_init(bar(B_Q_EMPTY + b), 1);
+      mbar_init(bar(B_S_FULL + b), 1); mbar_init(bar(B_P_FULL + b), kSoftmaxThreads);
+      mbar_init(bar(B_O_FULL + b), 1);
+    }
+    mbar_init(bar(B_GROUP), kSoftmaxThreads);
+    *s_abort = 0;
+    *s_dummy = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int x = tid; x <= n_bs; x += kThreads) s_tile[x] = ws_ptr<int>(a.ws, L.tile_prefix)[x];
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
+                 ::"r"(smem_u32(s_tmem)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (warp == 4 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+
+  const long long T = (long long)s_tile[n_bs] * n_kv;
+  // with fewer tiles than CTAs only the first T CTAs get a (one-tile) slice, so
+  // that every CTA in [0, C) has work and the per-pair contributor count is exact
+  const int C = (int)min((long long)gridDim.x, T);
+  const long long sl_begin = c < C ? slice_begin(c, T, C) : 0;
+  const long long sl_end = c < C ? slice_begin(c + 1, T, C) : 0;
+  const int* kv_len = ws_ptr<int>(a.ws, L.kv_len);
+
+  if (warp == 4) {
+    // ===================================================== TMA producer warp
+    Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
+    Segment sg;
+    unsigned u = 0;            // ring sequence number: K of tile it -> 2 it, V -> 2 it + 1
+    int seg = 0;
+    bool ok = true;
+    while (ok && sch.next(sg)) {
+      const int qb = seg & 1;
+      ok = mbar_wait(bar(B_Q_EMPTY + qb), ((seg >> 1) & 1) ^ 1, s_abort);
+      if (!ok) break;
+      if (lane == 0) {
+        const int row0 = ws_ptr<int>(a.ws, L.offset)[sg.i];
+        mbar_expect_tx(bar(B_Q_FULL + qb), kQBytes);
+        tma_load_4d(base + kOffQ + qb * kQBytes, &tm_q, bar(B_Q_FULL + qb), 0, 0, sg.g * 4, row0);
+        tma_load_4d(base + kOffQ + qb * kQBytes + kQBytes / 2, &tm_q, bar(B_Q_FULL + qb), 0, 1,
+                    sg.g * 4, row0);
+      }
+      const int len = kv_len[sg.i];
+      const int* bt = a.block_table + (size_t)sg.i * a.max_pages;
+      // lane l copies page l / 2, column half l % 2 (lanes 0..15)
+      const int pg_l = lane >> 1, half = lane & 1;
+      auto fetch_page = [&](int t) -> int {
+        const int p = t * (kTileTok / kPage) + pg_l;
+        int id = 0;
+        if (lane < 16 && p * kPage < len) {
+          id = bt[p];
+          if (id < 0 || id >= a.num_pages) { atomicOr(&hdr[H_STATUS], 2); id = 0; }
+        }
+        return id;
+      };
+      int page_next = fetch_page(sg.t0);
+      for (int t = sg.t0; t < sg.t1 && ok; ++t) {
+        const int page = page_next;
+        if (t + 1 < sg.t1) page_next = fetch_page(t + 1);
+        const int valid_tok = min(kTileTok, len - t * kTileTok);
+        const int n_pages = (valid_tok + kPage - 1) / kPage;
+#pragma unroll
+        for (int which = 0; which < 2; ++which, ++u) {
+          const int slot = u % kStages;
+          ok = mbar_wait(bar(B_KV_EMPTY + slot), ((u / kStages) & 1) ^ 1, s_abort);
+          if (!ok) break;
+          if (lane == 0) mbar_expect_tx(bar(B_KV_FULL + slot), n_pages * 2 * kPageBoxBytes);
+          __syncwarp();
+          if (lane < 16 && pg_l < n_pages) {
+            tma_load_5d(base + kOffKV + slot * kSlotBytes + half * kHalfSlot + pg_l * kPageBoxBytes,
+                        which == 0 ? &tm_k : &tm_v, bar(B_KV_FULL + slot), 0, half, 0, sg.g, page);
+          }
+        }
+      }
+      ++seg;
+    }
+    // on an aborted run, let the copies already issued land before the CTA's
+    // shared memory is released (bounded, like every other wait)
+    if (!ok) {
+      for (unsigned v = (u > kStages ? u - kStages : 0); v < u; ++v)
+        mbar_wait(bar(B_KV_FULL + v % kStages), (v / kStages) & 1, s_dummy);
+    }
+  } else if (warp == 5) {
+    // ============================================================ MMA issuer
+    if (lane == 0) {
+      Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
+      Segment sg;
+      unsigned it = 0;
+      int seg = 0;
+      bool ok = true;
+      auto issue_pv = [&](unsigned pt) -> bool {
+        const int b = pt & 1;
+        const unsigned uv = 2 * pt + 1;
+        const int slot = uv % kStages;
+        if (!mbar_wait(bar(B_P_FULL + b), (pt >> 1) & 1, s_abort)) return false;
+        if (!mbar_wait(bar(B_KV_FULL + slot), (uv / kStages) & 1, s_abort)) return false;
+        tc_fence_after();
+        const uint32_t p_base = base + kOffP + b * kPBytes;
+        const uint32_t v_base = base + kOffKV + slot * kSlotBytes;
+#pragma unroll
+        for (int kk = 0; kk < kTileTok / 16; ++kk) {
+          // A = P [64 rows][128 tok] K-major: 64-token blocks of 8 KB, 32 B per 16 tokens
+          const uint64_t ad = smem_desc(p_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
+          // B = V [128 tok][128 d] with d contiguous: MN-major, 16 tokens = 2 KB
+          const uint64_t bd = smem_desc(v_base + kk * (16 * 128), kHalfSlot, 1024);
+          umma(tmem + 256 + b * 128, ad, bd, kIdescPV, kk > 0);
+        }
+        umma_commit(bar(B_O_FULL + b));
+        umma_commit(bar(B_KV_EMPTY + slot));
+        return true;
+      };
+      while (ok && sch.next(sg)) {
+        const int qb = seg & 1;
+        ok = mbar_wait(bar(B_Q_FULL + qb), (seg >> 1) & 1, s_abort);
+        for (int t = sg.t0; t < sg.t1 && ok; ++t, ++it) {
+          const int b = it & 1;
+          const unsigned uk = 2 * it;
+          const int slot = uk % kStages;
+          ok = mbar_wait(bar(B_KV_FULL + slot), (uk / kStages) & 1, s_abort);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t q_base = base + kOffQ + qb * kQBytes;
+          const uint32_t k_base = base + kOffKV + slot * kSlotBytes;
+#pragma unroll
+          for (int kk = 0; kk < kD / 16; ++kk) {
+            const uint64_t ad = smem_desc(q_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
+            const uint64_t bd = smem_desc(k_base + (kk >> 2) * kHalfSlot + (kk & 3) * 32, 16, 1024);
+            umma(tmem + b * 128, ad, bd, kIdescS, kk > 0);
+          }
+          umma_commit(bar(B_S_FULL + b));
+          umma_commit(bar(B_KV_EMPTY + slot));
+          if (t + 1 == sg.t1) umma_commit(bar(B_Q_EMPTY + qb));
+          if (it >= 1) ok = issue_pv(it - 1);
+        }
+        ++seg;
+      }
+      if (ok && it >= 1) ok = issue_pv(it - 1);
+    }
+    __syncwarp();
+  } else {
+    // ====================================================== softmax warps 0-3
+    // rows of capacity beyond M_live are written as zero, spread over the grid
+    {
+      const int m_live = hdr[H_M_LIVE];
+      const long long n16 = (long long)(kHalfW * n_bs - m_live) * Hq * (kD * 2 / 16);
+      uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.out) +
+                                            (size_t)m_live * Hq * kD);
+      for (long long x = (long long)c * kSoftmaxThreads + tid; x < n16;
+           x += (long long)gridDim.x * kSoftmaxThreads)
+        dst[x] = make_uint4(0, 0, 0, 0);
+    }
+    const int row = warp * 16 + lane;                 // tile row m = 4 j + h_local
+    const int j_row = row >> 2, h_loc = row & 3;
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    const float scale_log2 = a.sm_scale * 1.4426950408889634f;
+    float* part_o = ws_ptr<float>(a.ws, L.part_o);
+    float* part_ml = ws_ptr<float>(a.ws, L.part_ml);
+    int* pair_cnt = ws_ptr<int>(a.ws, L.pair_cnt);
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a.out);
+
+    Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
+    Segment sg;
+    unsigned it = 0;
+    bool ok = true;
+    float acc[kD];
+    // bounded barrier among the 128 softmax threads (an mbarrier, so that a
+    // thread that gave up cannot leave the others stuck)
+    unsigned group_phase = 0;
+    auto group_sync = [&]() -> bool {
+      mbar_arrive(bar(B_GROUP));
+      const bool r = mbar_wait(bar(B_GROUP), group_phase & 1, s_abort);
+      ++group_phase;
+      return r;
+    };
+    while (ok && sch.next(sg)) {
+      const int ki = ws_ptr<int>(a.ws, L.k)[sg.i];
+      const int oi = ws_ptr<int>(a.ws, L.offset)[sg.i];
+      const int len = kv_len[sg.i];
+      const bool live = lane < 16 && j_row < ki;
+      const int pos = live ? ws_ptr<int>(a.ws, L.positions)[oi + j_row] : -1;
+      float m_run = -INFINITY, l_run = 0.0f, alpha_pending = 0.0f;
+#pragma unroll
+      for (int d = 0; d < kD; ++d) acc[d] = 0.0f;
+
+      auto fold_o = [&](unsigned pt) -> bool {       // acc = acc * alpha + O_pt
+        const int b = pt & 1;
+        if (!mbar_wait(bar(B_O_FULL + b), (pt >> 1) & 1, s_abort)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          float o[32];
+          tmem_ld32(t_lane + 256 + b * 128 + ch * 32, o);
+#pragma unroll
+          for (int x = 0; x < 32; ++x) acc[ch * 32 + x] = fmaf(acc[ch * 32 + x], alpha_pending, o[x]);
+        }
+        tc_fence_before();
+        return true;
+      };
+
+      for (int t = sg.t0; t < sg.t1 && ok; ++t, ++it) {
+        const int b = it & 1;
+        ok = mbar_wait(bar(B_S_FULL + b), (it >> 1) & 1, s_abort);
+        if (!ok) break;
+        tc_fence_after();
+        const int vis = min(kTileTok, max(0, pos + 1 - t * kTileTok));   // visible columns of this row
+        const uint32_t s_addr = t_lane + b * 128;
+        // pass 1: row maximum over the visible columns
+        float mx = -INFINITY;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          float s[32];
+          tmem_ld32(s_addr + ch * 32, s);
+          if (live) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) mx = (ch * 32 + x < vis) ? fmaxf(mx, s[x]) : mx;
+          }
+        }
+        const float m_new = fmaxf(m_run, mx * scale_log2);
+        const float m_safe = (m_new == -INFINITY) ? 0.0f : m_new;
+        const float alpha = ex2(m_run - m_safe);
+        // the previous use of this P buffer (tile it - 2) was consumed by an MMA
+        // whose completion this thread already saw (o_full of it - 2)
+        const uint32_t p_row = base + kOffP + b * kPBytes + row * 128;
+        float psum = 0.0f;
+        // pass 2: p = exp2(s * scale - m), bf16, swizzled store
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          float s[32];
+          tmem_ld32(s_addr + ch * 32, s);
+          if (live) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int x = 0; x < 32; x += 2) {
+              const int col = ch * 32 + x;
+              float p0 = ex2(fmaf(s[x], scale_log2, -m_safe));
+              float p1 = ex2(fmaf(s[x + 1], scale_log2, -m_safe));
+              p0 = (col < vis) ? p0 : 0.0f;
+              p1 = (col + 1 < vis) ? p1 : 0.0f;
+              psum += p0 + p1;
+              pk[x >> 1] = pack_bf16(p0, p1);
+            }
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              const int chunk = ch * 4 + q4;                       // 16-byte chunk = 8 tokens
+              const uint32_t addr = p_row + (chunk >> 3) * (kTcRows * 128) +
+                                    (((chunk & 7) ^ (row & 7)) << 4);
+              st_shared_v4(addr, pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
+            }
+          }
+        }
+        if (live) { l_run = l_run * alpha + psum; m_run = m_new; }
+        // last tile of the pair: V rows at or beyond the request's key count
+        // must be finite (0 x NaN would poison the row): zero them once the
+        // copy has landed
+        if (t + 1 == sg.n_tiles && len - t * kTileTok < kTileTok) {
+          const unsigned uv = 2 * it + 1;
+          const int slot = uv % kStages;
+          ok = mbar_wait(bar(B_KV_FULL + slot), (uv / kStages) & 1, s_abort);
+          if (!ok) break;
+          const int first = len - t * kTileTok;                    // first invalid token row
+          const int n_chunks = (kTileTok - first) * 16;            // 16-byte chunks, both halves
+          const uint32_t v_base = base + kOffKV + slot * kSlotBytes;
+          for (int x = tid; x < n_chunks; x += kSoftmaxThreads) {
+            const int r = first + (x >> 4), hc = x & 15;
+            st_shared_v4(v_base + (hc >> 3) * kHalfSlot + r * 128 + ((hc & 7) << 4), 0, 0, 0, 0);
+          }
+        }
+        tc_fence_before();
+        fence_async_smem();
+        mbar_arrive(bar(B_P_FULL + b));
+        if (t > sg.t0) ok = fold_o(it - 1);
+        alpha_pending = alpha;
+      }
+      if (!ok) break;
+      ok = fold_o(it - 1);                              // drain the last tile of the run
+      if (!ok) break;
+
+      const bool whole = (sg.t0 == 0 && sg.t1 == sg.n_tiles);
+      bool write_rows = whole;
+      if (!whole) {
+        // un-normalised partial to the workspace, then the pair's ticket
+        const int slot_id = c * 2 + (sg.first_of_cta ? 0 : 1);
+        if (live) {
+          float4* po = reinterpret_cast<float4*>(part_o + ((size_t)slot_id * kTcRows + row) * kD);
+#pragma unroll
+          for (int d = 0; d < kD; d += 4) po[d >> 2] = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
+          part_ml[((size_t)slot_id * kTcRows + row) * 2] = m_run;
+          part_ml[((size_t)slot_id * kTcRows + row) * 2 + 1] = l_run;
+        }
+        __threadfence();
+        if (!group_sync()) { ok = false; break; }
+        const long long p0 = ((long long)s_tile[sg.i] * n_kv) + (long long)sg.g * sg.n_tiles;
+        const int c_lo = cta_of(p0, T, C), c_hi = cta_of(p0 + sg.n_tiles - 1, T, C);
+        if (tid == 0) {
+          const int old = atomicAdd(&pair_cnt[sg.i * n_kv + sg.g], 1);
+          *s_ticket = (old == c_hi - c_lo);
+          if (old == c_hi - c_lo) pair_cnt[sg.i * n_kv + sg.g] = 0;   // ready for the next launch
+        }
+        if (!group_sync()) { ok = false; break; }
+        if (*s_ticket) {
+          __threadfence();
+          write_rows = true;
+          if (live) {
+            for (int cc = c_lo; cc <= c_hi; ++cc) {
+              if (cc == c) continue;
+              const int sid = cc * 2 + (slice_begin(cc, T, C) >= p0 ? 0 : 1);
+              const float m_o = __ldcg(&part_ml[((size_t)sid * kTcRows + row) * 2]);
+              const float l_o = __ldcg(&part_ml[((size_t)sid * kTcRows + row) * 2 + 1]);
+              const float m_tot = fmaxf(m_run, m_o);
+              const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
+              const float w_me = ex2(m_run - m_s), w_o = ex2(m_o - m_s);
+              const float4* po = reinterpret_cast<const float4*>(part_o + ((size_t)sid * kTcRows + row) * kD);
+#pragma unroll
+              for (int d = 0; d < kD; d += 4) {
+                const float4 v = __ldcg(&po[d >> 2]);
+                acc[d] = acc[d] * w_me + v.x * w_o;
+                acc[d + 1] = acc[d + 1] * w_me + v.y * w_o;
+                acc[d + 2] = acc[d + 2] * w_me + v.z * w_o;
+                acc[d + 3] = acc[d + 3] * w_me + v.w * w_o;
+              }
+              l_run = l_run * w_me + l_o * w_o;
+              m_run = m_tot;
+            }
+          }
+        }
+        if (!group_sync()) { ok = false; break; }            // s_ticket is reused by the next run
+      }
+      if (write_rows && live) {
+        const float inv = 1.0f / l_run;
+        uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(oi + j_row) * Hq + sg.g * 4 + h_loc) * kD);
+#pragma unroll
+        for (int d = 0; d < kD; d += 8) {
+          dst[d >> 3] = make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv),
+                                   pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
+                                   pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv),
+                                   pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && *s_abort) atomicOr(&hdr[H_STATUS], 8 /*TIMEOUT*/);
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
+// ------------------------------------------------------------ host: tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+struct MapKey {
+  const void* ptr; int a, b;
+  bool operator<(const MapKey& o) const {
+    return ptr != o.ptr ? ptr < o.ptr : (a != o.a ? a < o.a : b < o.b);
+  }
+};
+std::mutex g_map_mu;
+std::map<MapKey, CUtensorMap> g_kv_maps, g_q_maps;
+
+// K or V of one layer: [num_pages][n_kv][16 tok][128 d] viewed as
+// (d_lo 64, d_hi 2, tok 16, head, page); one box = one page-head, 64 columns
+bool kv_map(const void* ptr, int n_kv, int num_pages, CUtensorMap* out) {
+  std::lock_guard<std::mutex> lk(g_map_mu);
+  MapKey key{ptr, n_kv, num_pages};
+  auto it = g_kv_maps.find(key);
+  if (it != g_kv_maps.end()) { *out = it->second; return true; }
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[5] = {64, 2, (cuuint64_t)kPage, (cuuint64_t)n_kv, (cuuint64_t)num_pages};
+  cuuint64_t strides[4] = {128, 256, (cuuint64_t)kPage * kD * 2, (cuuint64_t)n_kv * kPage * kD * 2};
+  cuuint32_t box[5] = {64, 1, (cuuint32_t)kPage, 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides,
+                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (g_kv_maps.size() > 4096) g_kv_maps.clear();
+  g_kv_maps[key] = *out;
+  return true;
+}
+
+// q: [rows][n_q][128] viewed as (d_lo 64, d_hi 2, head, row); box = 4 heads x 16 rows
+bool q_map(const void* ptr, int n_q, int rows, CUtensorMap* out) {
+  std::lock_guard<std::mutex> lk(g_map_mu);
+  MapKey key{ptr, n_q, rows};
+  auto it = g_q_maps.find(key);
+  if (it != g_q_maps.end()) { *out = it->second; return true; }
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[4] = {64, 2, (cuuint64_t)n_q, (cuuint64_t)rows};
+  cuuint64_t strides[3] = {128, (cuuint64_t)kD * 2, (cuuint64_t)n_q * kD * 2};
+  cuuint32_t box[4] = {64, 1, 4, 16};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides,
+                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (g_q_maps.size() > 4096) g_q_maps.clear();
+  g_q_maps[key] = *out;
+  return true;
+}
+
+}  // namespace
+
+cudaError_t attn_tc_prepare() {
+  return cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kSmemBytes);
+}
+
+cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t stream) {
+  WsLayout L = ws_layout(a.n_bs, a.n_kv_heads, a.num_ctas);
+  CUtensorMap tq, tk, tv;
+  if (!q_map(a.q, a.n_q_heads, kHalfW * a.n_bs, &tq) ||
+      !kv_map(a.k_cache, a.n_kv_heads, a.num_pages, &tk) ||
+      !kv_map(a.v_cache, a.n_kv_heads, a.num_pages, &tv))
+    return cudaErrorNotSupported;
+  attn_tc_kernel<<<a.num_ctas, kThreads, kSmemBytes, stream>>>(a, L, tq, tk, tv);
+  return cudaGetLastError();
+}
+
+}  // namespace dscale

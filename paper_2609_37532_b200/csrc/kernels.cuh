@@ -1,0 +1,61 @@
+// Internal launch interface between api.cu and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "ws_layout.cuh"
+
+namespace dscale {
+
+struct AllocArgs {
+  void* ws;
+  int n_bs;
+  const int32_t* n_live;
+  const float* scores;
+  int scores_are_logits;
+  const int32_t* draft_tokens;
+  const int32_t* ctx_len;
+  const int32_t* block_table;
+  int max_pages;
+  int num_pages;
+  int n_kv_heads;
+  int num_ctas;
+};
+cudaError_t launch_alloc(const AllocArgs& a, cudaStream_t stream);
+
+struct AcceptArgs {
+  void* ws;
+  int n_bs;
+  const float* logits;
+  int64_t ld;
+  int vocab;
+  int32_t* accept_len;
+  int32_t* next_anchor;
+  int32_t* out_tokens;
+  int32_t* out_len;
+  int32_t* ctx_len_inout;
+  int n_kv_heads;
+  int num_ctas;
+};
+cudaError_t launch_accept(const AcceptArgs& a, cudaStream_t stream);
+
+struct AttnArgs {
+  void* ws;
+  int n_bs;
+  const void* q;
+  const void* k_cache;
+  const void* v_cache;
+  const int32_t* block_table;
+  int max_pages;
+  int num_pages;
+  int n_q_heads;
+  int n_kv_heads;
+  float sm_scale;
+  void* out;
+  int num_ctas;
+};
+cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t stream);
+// returns cudaErrorNotSupported if the driver entry point for tensor maps is missing
+cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t stream);
+
+}  // namespace dscale

@@ -1,0 +1,75 @@
+// Fixed-address workspace layout (the paper's buffer_bs, Eq. 12).
+//
+// The caller allocates one block of device memory per captured capacity n_bs;
+// every stage reads and writes its sections at offsets that depend only on
+// (n_bs, n_kv_heads, num_ctas), so addresses and shapes never change between
+// graph replays.  The int32 index sections come first and depend on n_bs
+// alone, which is what dscale_ws_field relies on.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+
+namespace dscale {
+
+constexpr int kW = 16;            // verification slots per request (anchor + 15 candidates)
+constexpr int kHalfW = 8;         // budget per live request (Eq. 3)
+constexpr int kPage = 16;         // tokens per KV page
+constexpr int kD = 128;           // head_dim
+constexpr int kMaxNbs = 64;
+constexpr int kTileTok = 128;     // keys per attention tile (8 pages)
+constexpr int kAccMaxChunks = 16; // vocab chunks per row in the argmax
+constexpr int kTcRows = 64;       // rows of the tensor-core query tile (GQA group 4 x 16 slots)
+
+// header words (int32)
+enum HdrWord {
+  H_STATUS = 0, H_N_LIVE = 1, H_M_LIVE = 2, H_TOTAL_TILES = 3, H_ACCEPT_TICKET = 4,
+  H_MAGIC = 5, H_WORDS = 64
+};
+
+struct WsLayout {
+  size_t hdr, k, k0, offset, q_start, q_end, tokens, positions, kv_refs, row_req, top1,
+      kv_len, tile_prefix, qscores, amax_val, amax_idx, pair_cnt, part_o, part_ml, total;
+};
+
+__host__ __device__ inline size_t ws_align(size_t x) { return (x + 255) & ~size_t(255); }
+
+__host__ __device__ inline WsLayout ws_layout(int n_bs, int n_kv_heads, int num_ctas) {
+  WsLayout L;
+  size_t o = 0;
+  const size_t m_bs = size_t(kHalfW) * n_bs;
+  L.hdr = o;         o = ws_align(o + H_WORDS * 4);
+  L.k = o;           o = ws_align(o + n_bs * 4);
+  L.k0 = o;          o = ws_align(o + n_bs * 4);
+  L.offset = o;      o = ws_align(o + (n_bs + 1) * 4);
+  L.q_start = o;     o = ws_align(o + n_bs * 4);
+  L.q_end = o;       o = ws_align(o + n_bs * 4);
+  L.tokens = o;      o = ws_align(o + m_bs * 4);
+  L.positions = o;   o = ws_align(o + m_bs * 4);
+  L.kv_refs = o;     o = ws_align(o + m_bs * 4);
+  L.row_req = o;     o = ws_align(o + m_bs * 4);
+  L.top1 = o;        o = ws_align(o + m_bs * 4);
+  L.kv_len = o;      o = ws_align(o + n_bs * 4);
+  L.tile_prefix = o; o = ws_align(o + (n_bs + 1) * 4);
+  L.qscores = o;     o = ws_align(o + size_t(n_bs) * kW * 4);
+  L.amax_val = o;    o = ws_align(o + m_bs * kAccMaxChunks * 4);
+  L.amax_idx = o;    o = ws_align(o + m_bs * kAccMaxChunks * 4);
+  L.pair_cnt = o;    o = ws_align(o + size_t(n_bs) * n_kv_heads * 4);
+  // split-KV partials of the attention kernel: per CTA two slots (the segment
+  // that starts its range and the one that ends it), each kTcRows rows of
+  // (128 fp32 accumulators) plus (row max, row sum)
+  L.part_o = o;      o = ws_align(o + size_t(num_ctas) * 2 * kTcRows * kD * 4);
+  L.part_ml = o;     o = ws_align(o + size_t(num_ctas) * 2 * kTcRows * 2 * 4);
+  L.total = o;
+  return L;
+}
+
+template <typename T>
+__host__ __device__ inline T* ws_ptr(void* ws, size_t off) {
+  return reinterpret_cast<T*>(reinterpret_cast<char*>(ws) + off);
+}
+template <typename T>
+__host__ __device__ inline const T* ws_ptr(const void* ws, size_t off) {
+  return reinterpret_cast<const T*>(reinterpret_cast<const char*>(ws) + off);
+}
+
+}  // namespace dscale
