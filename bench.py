@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the packed verify step (allocation -> attention x L -> acceptance).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over one batch of seeded synthetic
+input, replayed as ONE captured CUDA graph.  The default workload is the
+Qwen3-8B-shaped full step at concurrency 32 (36 layers, contexts 2048-8192).
+Prints one JSON line (rank 0).  With N > 1 (launched by torch.distributed.run)
+every rank runs an independent replica on its own GPU with its own batch:
+the path shards by request and needs no collective, so scaling is weak.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from dscale_inputs import (CONFIGS, make_kv_layer, make_logits_unpacked, make_q_unpacked,  # noqa: E402
+                           make_requests, rows_to_packed, small_variant)
+
+SCALE = 1.0 / float(np.sqrt(128.0))
+METRIC = "verified_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# --------------------------------------------------------------------- helpers
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def recorded_traffic(workload: str):
+    """DRAM bytes per attention launch from the committed ncu summary, if any."""
+    p = os.path.join(ROOT, "profiles", "attn_tc_traffic.json")
+    if os.path.exists(p):
+        try:
+            return json.load(open(p)).get(workload)
+        except Exception:
+            return None
+    return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+def algorithmic_bytes(cfg, req, k):
+    """Bytes the method must move: per layer K and V of every visible key, the
+    page ids, Q in and O out; per step the logits, scores and packed fields."""
+    n = req["n_live"]
+    kv_len = req["ctx_len"][:n].astype(np.int64) + np.asarray(k[:n], dtype=np.int64)
+    kv = int(kv_len.sum()) * cfg.n_kv_heads * 128 * 2 * 2
+    pages = int(((kv_len + 15) // 16).sum()) * 4
+    qo = 2 * 8 * n * cfg.n_q_heads * 128 * 2
+    per_layer = kv + pages + qo
+    logits = 8 * n * cfg.vocab * 4
+    small = n * 15 * 4 + n * 16 * 4 + 4 * 8 * n * 4 + n * 19 * 4
+    return per_layer, logits + small
+
+
+# ------------------------------------------------------------------ CPU oracle
+def oracle_step_sample(cfg, req, kc0, vc0, q0_unpacked, logits_unpacked):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload:
+    allocation and acceptance in full, attention on ONE layer (all requests),
+    and extrapolates the step time to cfg.layers layers.  Returns
+    (tokens_per_s, seconds of CPU work, description)."""
+    from oracle import accept as OC
+    from oracle import dvl_alloc as OA
+    from oracle import verify_attn as OV
+    t0 = time.perf_counter()
+    alloc = OA.dvl_alloc(req["n_bs"], req["n_live"], req["scores"], req["draft_tokens"],
+                         req["ctx_len"], req["block_table"])
+    t1 = time.perf_counter()
+    qp = rows_to_packed(q0_unpacked, alloc["k"], alloc["offset"], req["n_live"], 8 * req["n_bs"])
+    lp = rows_to_packed(logits_unpacked, alloc["k"], alloc["offset"], req["n_live"], 8 * req["n_bs"])
+    qf, kf, vf, lf = qp.float().numpy(), kc0.float().numpy(), vc0.float().numpy(), lp.numpy()
+    t2 = time.perf_counter()
+    OV.verify_attn(qf, kf, vf, req["block_table"], req["ctx_len"], alloc["k"], alloc["offset"],
+                   req["n_live"], cfg.n_q_heads, cfg.n_kv_heads, SCALE)
+    t3 = time.perf_counter()
+    res = OC.accept(lf, cfg.vocab, alloc["tokens"], alloc["k"], alloc["offset"], req["n_live"],
+                    req["n_bs"])
+    t4 = time.perf_counter()
+    tokens = int(res["out_len"].sum())
+    step = (t1 - t0) + cfg.layers * (t3 - t2) + (t4 - t3)
+    work = (t1 - t0) + (t3 - t2) + (t4 - t3)
+    desc = (f"allocation and acceptance in full, attention on layer 0 of {cfg.layers} "
+            f"(all {req['n_live']} requests), attention time x {cfg.layers}")
+    return tokens / step, work, desc
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, rank):
+    """Reference arm: the CPU oracle timed on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    cfg = CONFIGS[args.workload]
+    req = make_requests(cfg)
+    kc, vc = make_kv_layer(req, 0, poison=False)
+    qu = make_q_unpacked(req, 0)
+    lu = make_logits_unpacked(req)
+    vals, work = [], 0.0
+    desc = ""
+    for s in range(args.warmup + args.steps):
+        v, w, desc = oracle_step_sample(cfg, req, kc, vc, qu, lu)
+        if s >= args.warmup:
+            vals.append(v); work += w
+    value = float(np.mean(vals))
+    cores = blas_threads()
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * work / max(1, args.steps), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "requests": cfg.n, "layers": cfg.layers,
+                   "ctx": [cfg.ctx_lo, cfg.ctx_hi], "vocab": cfg.vocab},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------- GPU bench
+def run_ours(args, rank, world, local_rank):
+    import paper_2609_37532_b200 as P
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    base = CONFIGS[args.workload]
+    cfg = small_variant(base, seed=base.seed + 1000 * rank)      # every replica has its own batch
+    if args.layers:
+        cfg = small_variant(cfg, layers=args.layers)
+    req = make_requests(cfg)
+    n_bs, n = req["n_bs"], req["n_live"]
+    ws = P.VerifyWorkspace(n_bs, cfg.n_q_heads, cfg.n_kv_heads, device=dev)
+
+    d_n_live = torch.tensor([n], dtype=torch.int32, device=dev)
+    d_scores = torch.as_tensor(req["scores"]).to(dev)
+    d_draft = torch.as_tensor(req["draft_tokens"]).to(dev)
+    d_ctx = torch.as_tensor(req["ctx_len"]).to(dev)
+    d_bt = torch.as_tensor(req["block_table"]).to(dev).contiguous()
+
+    def do_alloc():
+        P.alloc_verify(ws, d_n_live, d_scores, d_draft, d_ctx, d_bt, req["num_pages"])
+
+    do_alloc()
+    torch.cuda.synchronize()
+    k = ws.field("k").cpu().numpy().copy()
+    offset = ws.field("offset").cpu().numpy().copy()
+    assert int(k[:n].sum()) == 8 * n and ws.status() == 0
+
+    layers = []
+    for l in range(cfg.layers):
+        kc, vc = make_kv_layer(req, l, device=str(dev), poison=False)
+        qp = rows_to_packed(make_q_unpacked(req, l, device=str(dev)), k, offset, n, 8 * n_bs)
+        layers.append((qp.contiguous(), kc, vc, torch.empty_like(qp)))
+    lu = make_logits_unpacked(req, device=str(dev))
+    logits = rows_to_packed(lu, k, offset, n, 8 * n_bs).contiguous()
+    del lu
+    outs = [torch.zeros(n_bs, dtype=torch.int32, device=dev), torch.zeros(n_bs, dtype=torch.int32, device=dev),
+            torch.zeros((n_bs, 16), dtype=torch.int32, device=dev), torch.zeros(n_bs, dtype=torch.int32, device=dev)]
+
+    attn = P.verify_attn if args.attn == "tensor" else P.verify_attn_simt
+
+    def do_attn():
+        for (q, kc, vc, o) in layers:
+            attn(ws, q, kc, vc, d_bt, SCALE, o)
+
+    def do_accept():
+        P.accept(ws, logits, cfg.vocab, outs[0], outs[1], outs[2], outs[3], None)
+
+    def step_direct():
+        do_alloc(); do_attn(); do_accept()
+
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        step_direct()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            step_direct()
+    torch.cuda.synchronize()
+    tokens_per_step = int(outs[3].sum().item())
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            graph.replay()
+        barrier()
+        if rank == 0:
+            sampler.start()
+        # ---- timed region 1: K replays of the captured step (headline) ----
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(args.steps):
+            graph.replay()
+        e1.record(stream)
+        barrier()
+        ms_total = e0.elapsed_time(e1)
+
+        # ---- timed region 2: same steps as direct launches, with events around the
+        # attention launches, for the per-kernel roofline ----
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
+               torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for s in range(args.steps):
+            do_alloc()
+            ev[s][0].record(stream)
+            do_attn()
+            ev[s][1].record(stream)
+            do_accept()
+            ev[s][2].record(stream)
+        barrier()
+        attn_ms = float(np.mean([a.elapsed_time(b) for a, b, _ in ev])) / max(1, cfg.layers)
+        accept_ms = float(np.mean([b.elapsed_time(c) for _, b, c in ev]))
+
+        # ---- timed region 3: end to end through the host-buffer C ABI call ----
+        hs = P.HostStep(ws, req["max_pages"], req["num_pages"], layers, logits, cfg.vocab, SCALE)
+        hs.h_n_live[0] = n
+        hs.h_scores.copy_(torch.as_tensor(req["scores"]))
+        hs.h_draft.copy_(torch.as_tensor(req["draft_tokens"]))
+        hs.h_ctx_len.copy_(torch.as_tensor(req["ctx_len"]))
+        hs.h_block_table.copy_(torch.as_tensor(req["block_table"]))
+        for _ in range(max(1, args.warmup)):
+            hs.run(); stream.synchronize()
+        barrier()
+        t0 = time.perf_counter()
+        e2e_tokens = 0
+        for _ in range(args.steps):
+            hs.run()
+            stream.synchronize()                      # the caller reads the outputs every step
+            e2e_tokens += int(hs.h_out_len.sum())
+        e2e_s = time.perf_counter() - t0
+    clocks = sampler.stop() if rank == 0 else None
+    assert ws.status() == 0, f"device status {ws.status()}"
+
+    ms_step = ms_total / args.steps
+    t = torch.tensor([ms_step, attn_ms, e2e_s, float(tokens_per_step), float(e2e_tokens)],
+                     dtype=torch.float64, device=dev)
+    if dist is not None:
+        tmax = t.clone(); dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        tsum = t.clone(); dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+    else:
+        tmax = tsum = t
+    ms_step, attn_ms, e2e_s = float(tmax[0]), float(tmax[1]), float(tmax[2])
+    tokens_all, e2e_tokens_all = float(tsum[3]), float(tsum[4])
+    value = tokens_all / (ms_step * 1e-3)
+    e2e_value = e2e_tokens_all / e2e_s
+
+    if rank == 0:
+        per_layer_b, per_step_b = algorithmic_bytes(cfg, req, k)
+        peak, peak_kind = measured_peak()
+        achieved = per_layer_b / (attn_ms * 1e-3) / 1e9
+        step_gbs = (per_layer_b * cfg.layers + per_step_b) / (ms_step * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "requests_per_gpu": n, "layers": cfg.layers,
+                       "heads": [cfg.n_q_heads, cfg.n_kv_heads], "ctx": [cfg.ctx_lo, cfg.ctx_hi],
+                       "vocab": cfg.vocab, "packed_rows": 8 * n, "attn": args.attn,
+                       "l2": "inputs_larger_than_L2 (%.1f GB per step)" %
+                             ((per_layer_b * cfg.layers + per_step_b) / 1e9),
+                       "launch": "one captured CUDA graph per step"},
+            "verified_tokens_per_step": tokens_per_step,
+            "packed_rows_per_s": 8 * n * world / (ms_step * 1e-3),
+            "step_gbs": step_gbs, "step_frac_of_peak": step_gbs / peak,
+            "step_frac_of_8tbs": step_gbs / 8000.0,
+            "roofline": {"bound": "hbm", "kernel": "attn_tc_kernel" if args.attn == "tensor" else "attn_simt_kernel",
+                         "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                         "frac": achieved / peak, "frac_of_8tbs": achieved / 8000.0,
+                         "bytes_per_launch": per_layer_b, "us_per_launch": attn_ms * 1e3,
+                         "traffic": recorded_traffic(cfg.name)},
+            "accept_us": accept_ms * 1e3,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": hs.h2d_bytes,
+                    "d2h_bytes_per_step": hs.d2h_bytes, "ms_per_step": 1e3 * e2e_s / args.steps,
+                    "api": "dscale_verify_step_host (pinned host inputs/outputs, KV/Q/logits resident)"},
+            "gpu_launches": args.steps * (P.lib.dscale_launches_per_call(0) +
+                                          cfg.layers * P.lib.dscale_launches_per_call(1 if args.attn == "tensor" else 3) +
+                                          P.lib.dscale_launches_per_call(2)),
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            kc0, vc0 = layers[0][1].cpu(), layers[0][2].cpu()
+            qu0 = make_q_unpacked(req, 0, device=str(dev)).cpu()
+            lu_cpu = make_logits_unpacked(req, device=str(dev)).cpu()
+            v, work, desc = oracle_step_sample(cfg, req, kc0, vc0, qu0, lu_cpu)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                    "sample": desc, "cpu_seconds": work}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen3_8b_step", choices=list(CONFIGS))
+    ap.add_argument("--attn", default="tensor", choices=["tensor", "simt"])
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local_rank = int(os.environ.get("LOCAL_RANK", 0))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -180,6 +180,40 @@ int dscale_accept(void* ws, int n_bs, const float* logits, int64_t ld, int vocab
                   int32_t* out_len, int32_t* ctx_len_inout, void* stream);
 
 /*
+ * One whole verify step driven from HOST buffers: what Algorithm 2 does between
+ * "stage inputs" and "read outputs" (lines 10-21).  The staged inputs
+ * (N, scores, draft tokens, context lengths, block table) are copied from host
+ * memory into `staging`, the three stages are enqueued (allocation, attention
+ * for each of n_layers layers, acceptance), and the outputs are copied back to
+ * host memory, all asynchronously on `stream`; the results are valid after the
+ * caller synchronises the stream.  Host buffers should be page-locked for the
+ * copies to be asynchronous.
+ *
+ *   h_*          HOST pointers, same shapes as in the per-stage calls
+ *   staging      DEVICE scratch of at least dscale_step_staging_bytes(n_bs, max_pages)
+ *                bytes, 256-byte aligned, owned by the caller, reused every step
+ *   layers       HOST array of n_layers entries of DEVICE pointers (q, k_cache,
+ *                v_cache, out of each layer; layouts as in dscale_verify_attn)
+ *   logits       DEVICE fp32 [8 n_bs][ld] (produced on the device by the LM head)
+ */
+typedef struct dscale_layer {
+  const void* q;
+  const void* k_cache;
+  const void* v_cache;
+  void* out;
+} dscale_layer;
+
+size_t dscale_step_staging_bytes(int n_bs, int max_pages);
+
+int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const float* h_scores,
+                            const int32_t* h_draft_tokens, const int32_t* h_ctx_len,
+                            const int32_t* h_block_table, int max_pages, int num_pages,
+                            void* staging, const dscale_layer* layers, int n_layers,
+                            int n_q_heads, int n_kv_heads, float sm_scale, const float* logits,
+                            int64_t ld, int vocab, int32_t* h_accept_len, int32_t* h_next_anchor,
+                            int32_t* h_out_tokens, int32_t* h_out_len, void* stream);
+
+/*
  * Device address of a workspace field (see DSCALE_WS_*), for tests and for
  * callers that feed packed fields to other kernels.  HOST call; returns NULL
  * for a bad field id.  The address depends only on (ws, n_bs).

@@ -5,8 +5,13 @@ torch tensors (device memory, streams) into the C ABI declared in
 include/dscale.h.  There is no CPU fallback: importing the binding without the
 built library raises.
 """
-from .binding import (DScaleError, VerifyWorkspace, accept, alloc_verify, lib, verify_attn,
+from .build import build as _build
+
+_build()          # no-op when libdscale.so is newer than its sources; raises if nvcc fails
+
+from .binding import (  # noqa: E402
+    DScaleError, HostStep, VerifyWorkspace, accept, alloc_verify, lib, verify_attn,
                       verify_attn_simt, WS_FIELDS)
 
-__all__ = ["DScaleError", "VerifyWorkspace", "accept", "alloc_verify", "lib", "verify_attn",
+__all__ = ["DScaleError", "HostStep", "VerifyWorkspace", "accept", "alloc_verify", "lib", "verify_attn",
            "verify_attn_simt", "WS_FIELDS"]

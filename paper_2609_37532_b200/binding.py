@@ -28,6 +28,18 @@ for _name in ("dscale_verify_attn", "dscale_verify_attn_simt"):
     getattr(lib, _name).argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _f, _vp, _vp]
 lib.dscale_accept.restype = _i
 lib.dscale_accept.argtypes = [_vp, _i, _vp, _i64, _i, _vp, _vp, _vp, _vp, _vp, _vp]
+
+
+class LayerPtrs(C.Structure):
+    _fields_ = [("q", _vp), ("k_cache", _vp), ("v_cache", _vp), ("out", _vp)]
+
+
+lib.dscale_step_staging_bytes.restype = _sz
+lib.dscale_step_staging_bytes.argtypes = [_i, _i]
+lib.dscale_verify_step_host.restype = _i
+lib.dscale_verify_step_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _i, _vp,
+                                        C.POINTER(LayerPtrs), _i, _i, _i, _f, _vp, _i64, _i,
+                                        _vp, _vp, _vp, _vp, _vp]
 lib.dscale_ws_field.restype = _vp
 lib.dscale_ws_field.argtypes = [_vp, _i, _i]
 lib.dscale_launches_per_call.restype = _i
@@ -140,3 +152,48 @@ def accept(ws, logits, vocab: int, accept_len, next_anchor, out_tokens, out_len,
     _check(lib.dscale_accept(C.c_void_p(ws.ptr), ws.n_bs, _ptr(logits), logits.stride(0), vocab,
                              _ptr(accept_len), _ptr(next_anchor), _ptr(out_tokens), _ptr(out_len),
                              _ptr(ctx_len_inout), _stream()), "dscale_accept")
+
+
+class HostStep:
+    """Whole verify step from pinned host buffers (dscale_verify_step_host).
+
+    Holds the pinned input / output buffers, the device staging scratch and
+    the per-layer pointer table; `run()` enqueues one step on the current
+    stream and returns without synchronising."""
+
+    def __init__(self, ws: VerifyWorkspace, max_pages: int, num_pages: int, layers, logits,
+                 vocab: int, sm_scale: float):
+        n_bs = ws.n_bs
+        self.ws, self.max_pages, self.num_pages = ws, max_pages, num_pages
+        self.vocab, self.sm_scale, self.logits = vocab, float(sm_scale), logits
+        pin = dict(pin_memory=True)
+        self.h_n_live = torch.zeros(1, dtype=torch.int32, **pin)
+        self.h_scores = torch.zeros((n_bs, 15), dtype=torch.float32, **pin)
+        self.h_draft = torch.zeros((n_bs, 16), dtype=torch.int32, **pin)
+        self.h_ctx_len = torch.zeros(n_bs, dtype=torch.int32, **pin)
+        self.h_block_table = torch.zeros((n_bs, max_pages), dtype=torch.int32, **pin)
+        self.h_accept_len = torch.zeros(n_bs, dtype=torch.int32, **pin)
+        self.h_next_anchor = torch.zeros(n_bs, dtype=torch.int32, **pin)
+        self.h_out_tokens = torch.zeros((n_bs, 16), dtype=torch.int32, **pin)
+        self.h_out_len = torch.zeros(n_bs, dtype=torch.int32, **pin)
+        nbytes = lib.dscale_step_staging_bytes(n_bs, max_pages)
+        self.staging = torch.empty(nbytes + 256, dtype=torch.uint8, device=ws.buf.device)
+        self.staging_ptr = self.staging.data_ptr() + (-self.staging.data_ptr()) % 256
+        self._keep = layers
+        self.table = (LayerPtrs * len(layers))()
+        for x, (q, kc, vc, out) in enumerate(layers):
+            _need(q, torch.bfloat16, "q"); _need(kc, torch.bfloat16, "k_cache")
+            _need(vc, torch.bfloat16, "v_cache"); _need(out, torch.bfloat16, "out")
+            self.table[x] = LayerPtrs(q.data_ptr(), kc.data_ptr(), vc.data_ptr(), out.data_ptr())
+        self.h2d_bytes = 4 + n_bs * (15 + 16 + 1 + max_pages) * 4
+        self.d2h_bytes = n_bs * (1 + 1 + 16 + 1) * 4
+
+    def run(self):
+        ws = self.ws
+        _check(lib.dscale_verify_step_host(
+            C.c_void_p(ws.ptr), ws.n_bs, _ptr(self.h_n_live), _ptr(self.h_scores),
+            _ptr(self.h_draft), _ptr(self.h_ctx_len), _ptr(self.h_block_table), self.max_pages,
+            self.num_pages, C.c_void_p(self.staging_ptr), self.table, len(self.table),
+            ws.n_q_heads, ws.n_kv_heads, self.sm_scale, _ptr(self.logits),
+            self.logits.stride(0), self.vocab, _ptr(self.h_accept_len), _ptr(self.h_next_anchor),
+            _ptr(self.h_out_tokens), _ptr(self.h_out_len), _stream()), "dscale_verify_step_host")

@@ -142,6 +142,85 @@ int dscale_accept(void* ws, int n_bs, const float* logits, int64_t ld, int vocab
   return launch_accept(a, (cudaStream_t)stream) == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
 }
 
+namespace {
+struct StagingLayout {
+  size_t n_live, scores, draft, ctx_len, block_table, accept_len, next_anchor, out_tokens,
+      out_len, total;
+};
+StagingLayout staging_layout(int n_bs, int max_pages) {
+  StagingLayout S;
+  size_t o = 0;
+  S.n_live = o;      o = ws_align(o + 4);
+  S.scores = o;      o = ws_align(o + size_t(n_bs) * 15 * 4);
+  S.draft = o;       o = ws_align(o + size_t(n_bs) * 16 * 4);
+  S.ctx_len = o;     o = ws_align(o + size_t(n_bs) * 4);
+  S.block_table = o; o = ws_align(o + size_t(n_bs) * max_pages * 4);
+  S.accept_len = o;  o = ws_align(o + size_t(n_bs) * 4);
+  S.next_anchor = o; o = ws_align(o + size_t(n_bs) * 4);
+  S.out_tokens = o;  o = ws_align(o + size_t(n_bs) * 16 * 4);
+  S.out_len = o;     o = ws_align(o + size_t(n_bs) * 4);
+  S.total = o;
+  return S;
+}
+}  // namespace
+
+size_t dscale_step_staging_bytes(int n_bs, int max_pages) {
+  if (n_bs < 1 || n_bs > DSCALE_MAX_NBS || max_pages < 1) return 0;
+  return staging_layout(n_bs, max_pages).total;
+}
+
+int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const float* h_scores,
+                            const int32_t* h_draft_tokens, const int32_t* h_ctx_len,
+                            const int32_t* h_block_table, int max_pages, int num_pages,
+                            void* staging, const dscale_layer* layers, int n_layers,
+                            int n_q_heads, int n_kv_heads, float sm_scale, const float* logits,
+                            int64_t ld, int vocab, int32_t* h_accept_len, int32_t* h_next_anchor,
+                            int32_t* h_out_tokens, int32_t* h_out_len, void* stream) {
+  if (!h_n_live || !h_scores || !h_draft_tokens || !h_ctx_len || !h_block_table || !staging ||
+      !layers || !h_accept_len || !h_next_anchor || !h_out_tokens || !h_out_len)
+    return DSCALE_ERR_INVALID_ARG;
+  if (n_bs < 1 || n_bs > DSCALE_MAX_NBS || max_pages < 1 || n_layers < 0 || !aligned(staging, 256))
+    return DSCALE_ERR_INVALID_ARG;
+  const StagingLayout S = staging_layout(n_bs, max_pages);
+  char* d = static_cast<char*>(staging);
+  cudaStream_t st = (cudaStream_t)stream;
+  auto h2d = [&](size_t off, const void* src, size_t bytes) {
+    return cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  };
+  auto d2h = [&](void* dst, size_t off, size_t bytes) {
+    return cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  };
+  if (!h2d(S.n_live, h_n_live, 4) || !h2d(S.scores, h_scores, size_t(n_bs) * 15 * 4) ||
+      !h2d(S.draft, h_draft_tokens, size_t(n_bs) * 16 * 4) ||
+      !h2d(S.ctx_len, h_ctx_len, size_t(n_bs) * 4) ||
+      !h2d(S.block_table, h_block_table, size_t(n_bs) * max_pages * 4))
+    return DSCALE_ERR_CUDA;
+  const int32_t* d_bt = reinterpret_cast<const int32_t*>(d + S.block_table);
+  int rc = dscale_alloc_verify(ws, n_bs, reinterpret_cast<const int32_t*>(d + S.n_live),
+                               reinterpret_cast<const float*>(d + S.scores), 0,
+                               reinterpret_cast<const int32_t*>(d + S.draft),
+                               reinterpret_cast<const int32_t*>(d + S.ctx_len), d_bt, max_pages,
+                               num_pages, stream);
+  if (rc != DSCALE_OK) return rc;
+  for (int l = 0; l < n_layers; ++l) {
+    rc = dscale_verify_attn(ws, n_bs, layers[l].q, layers[l].k_cache, layers[l].v_cache, d_bt,
+                            max_pages, num_pages, n_q_heads, n_kv_heads, sm_scale, layers[l].out,
+                            stream);
+    if (rc != DSCALE_OK) return rc;
+  }
+  rc = dscale_accept(ws, n_bs, logits, ld, vocab, reinterpret_cast<int32_t*>(d + S.accept_len),
+                     reinterpret_cast<int32_t*>(d + S.next_anchor),
+                     reinterpret_cast<int32_t*>(d + S.out_tokens),
+                     reinterpret_cast<int32_t*>(d + S.out_len), nullptr, stream);
+  if (rc != DSCALE_OK) return rc;
+  if (!d2h(h_accept_len, S.accept_len, size_t(n_bs) * 4) ||
+      !d2h(h_next_anchor, S.next_anchor, size_t(n_bs) * 4) ||
+      !d2h(h_out_tokens, S.out_tokens, size_t(n_bs) * 16 * 4) ||
+      !d2h(h_out_len, S.out_len, size_t(n_bs) * 4))
+    return DSCALE_ERR_CUDA;
+  return DSCALE_OK;
+}
+
 const int32_t* dscale_ws_field(const void* ws, int n_bs, int field) {
   if (!ws || n_bs < 1 || n_bs > DSCALE_MAX_NBS) return nullptr;
   const WsLayout L = ws_layout(n_bs, 1, 1);      // index sections depend on n_bs only
