@@ -27,11 +27,13 @@
 //              is signalled with tcgen05.commit on mbarriers.
 //   warps 0-3  softmax: thread (w, l < 16) owns row 16 w + l (TMEM lane 32 w + l),
 //              reads S with tcgen05.ld, keeps the running max / sum, writes P as
-//              bf16 into swizzled shared memory for the second MMA, and folds
-//              each per-tile product O_t (read back from TMEM) into fp32
-//              accumulators in registers, rescaled by exp2(m_old - m_new).
-// S and O_t are double-buffered in TMEM (4 x 128 columns), P and Q in shared
-// memory, so the MMA of tile t+1 overlaps the softmax of tile t.
+//              bf16 into swizzled shared memory for the second MMA.  O stays in
+//              TMEM for a whole run of tiles (the second MMA accumulates onto
+//              it); it is only rescaled in place when a row maximum outgrows its
+//              reference by 2^8, and read back once per run for the epilogue.
+// S is double-buffered in TMEM (2 x 128 columns) next to O (128 columns), P and
+// Q are double-buffered in shared memory, so the MMA of tile t+1 overlaps the
+// softmax of tile t.
 //
 // Every wait is bounded: when a wait runs out the CTA sets the TIMEOUT status
 // bit, stops issuing work, drains its outstanding copies and releases TMEM.
@@ -180,6 +182,29 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
   for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
+}
+__device__ __forceinline__ void tmem_ld128(uint32_t taddr, float* v) {
+  uint32_t r[128];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%128];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%129];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%64, %65, %66, %67, %68, %69, %70, %71, %72, %73, %74, %75, %76, %77, %78, %79, %80, %81, %82, %83, %84, %85, %86, %87, %88, %89, %90, %91, %92, %93, %94, %95}, [%130];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%96, %97, %98, %99, %100, %101, %102, %103, %104, %105, %106, %107, %108, %109, %110, %111, %112, %113, %114, %115, %116, %117, %118, %119, %120, %121, %122, %123, %124, %125, %126, %127}, [%131];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63]), "=r"(r[64]), "=r"(r[65]), "=r"(r[66]), "=r"(r[67]), "=r"(r[68]), "=r"(r[69]), "=r"(r[70]), "=r"(r[71]), "=r"(r[72]), "=r"(r[73]), "=r"(r[74]), "=r"(r[75]), "=r"(r[76]), "=r"(r[77]), "=r"(r[78]), "=r"(r[79]), "=r"(r[80]), "=r"(r[81]), "=r"(r[82]), "=r"(r[83]), "=r"(r[84]), "=r"(r[85]), "=r"(r[86]), "=r"(r[87]), "=r"(r[88]), "=r"(r[89]), "=r"(r[90]), "=r"(r[91]), "=r"(r[92]), "=r"(r[93]), "=r"(r[94]), "=r"(r[95]), "=r"(r[96]), "=r"(r[97]), "=r"(r[98]), "=r"(r[99]), "=r"(r[100]), "=r"(r[101]), "=r"(r[102]), "=r"(r[103]), "=r"(r[104]), "=r"(r[105]), "=r"(r[106]), "=r"(r[107]), "=r"(r[108]), "=r"(r[109]), "=r"(r[110]), "=r"(r[111]), "=r"(r[112]), "=r"(r[113]), "=r"(r[114]), "=r"(r[115]), "=r"(r[116]), "=r"(r[117]), "=r"(r[118]), "=r"(r[119]), "=r"(r[120]), "=r"(r[121]), "=r"(r[122]), "=r"(r[123]), "=r"(r[124]), "=r"(r[125]), "=r"(r[126]), "=r"(r[127])
+      : "r"(taddr), "r"(taddr + 32), "r"(taddr + 64), "r"(taddr + 96)
+      : "memory");
+#pragma unroll
+  for (int x = 0; x < 128; ++x) v[x] = __uint_as_float(r[x]);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+      ::"r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31])), "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() {
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -359,6 +384,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       unsigned it = 0;
       int seg = 0;
       bool ok = true;
+      bool first_of_run[2] = {true, true};   // per P buffer: does its tile start a run?
       auto issue_pv = [&](unsigned pt) -> bool {
         const int b = pt & 1;
         const unsigned uv = 2 * pt + 1;
@@ -374,7 +400,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           const uint64_t ad = smem_desc(p_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
           // B = V [128 tok][128 d] with d contiguous: MN-major, 16 tokens = 2 KB
           const uint64_t bd = smem_desc(v_base + kk * (16 * 128), kHalfSlot, 1024);
-          umma(tmem + 256 + b * 128, ad, bd, kIdescPV, kk > 0);
+          umma(tmem + 256, ad, bd, kIdescPV, (kk > 0) || !first_of_run[b]);
         }
         umma_commit(bar(B_O_FULL + b));
         umma_commit(bar(B_KV_EMPTY + slot));
@@ -385,6 +411,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         ok = mbar_wait(bar(B_Q_FULL + qb), (seg >> 1) & 1, s_abort);
         for (int t = sg.t0; t < sg.t1 && ok; ++t, ++it) {
           const int b = it & 1;
+          first_of_run[b] = (t == sg.t0);
           const unsigned uk = 2 * it;
           const int slot = uk % kStages;
           ok = mbar_wait(bar(B_KV_FULL + slot), (uk / kStages) & 1, s_abort);
@@ -423,6 +450,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     const int row = warp * 16 + lane;                 // tile row m = 4 j + h_local
     const int j_row = row >> 2, h_loc = row & 3;
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t o_addr = t_lane + 256;
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
     float* part_o = ws_ptr<float>(a.ws, L.part_o);
     float* part_ml = ws_ptr<float>(a.ws, L.part_ml);
@@ -433,7 +461,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     Segment sg;
     unsigned it = 0;
     bool ok = true;
-    float acc[kD];
     // bounded barrier among the 128 softmax threads (an mbarrier, so that a
     // thread that gave up cannot leave the others stuck)
     unsigned group_phase = 0;
@@ -443,83 +470,87 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       ++group_phase;
       return r;
     };
+    auto wait_pv = [&](unsigned pt) -> bool {        // P.V of tile pt has completed
+      return mbar_wait(bar(B_O_FULL + (pt & 1)), (pt >> 1) & 1, s_abort);
+    };
+
     while (ok && sch.next(sg)) {
       const int ki = ws_ptr<int>(a.ws, L.k)[sg.i];
       const int oi = ws_ptr<int>(a.ws, L.offset)[sg.i];
       const int len = kv_len[sg.i];
       const bool live = lane < 16 && j_row < ki;
       const int pos = live ? ws_ptr<int>(a.ws, L.positions)[oi + j_row] : -1;
-      float m_run = -INFINITY, l_run = 0.0f, alpha_pending = 0.0f;
-#pragma unroll
-      for (int d = 0; d < kD; ++d) acc[d] = 0.0f;
-
-      auto fold_o = [&](unsigned pt) -> bool {       // acc = acc * alpha + O_pt
-        const int b = pt & 1;
-        if (!mbar_wait(bar(B_O_FULL + b), (pt >> 1) & 1, s_abort)) return false;
-        tc_fence_after();
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          float o[32];
-          tmem_ld32(t_lane + 256 + b * 128 + ch * 32, o);
-#pragma unroll
-          for (int x = 0; x < 32; ++x) acc[ch * 32 + x] = fmaf(acc[ch * 32 + x], alpha_pending, o[x]);
-        }
-        tc_fence_before();
-        return true;
-      };
+      // O accumulates in TMEM relative to a reference maximum m_ref that is only
+      // raised (and O rescaled) when the row maximum outgrows it by 2^8
+      float m_ref = -INFINITY, l_run = 0.0f;
 
       for (int t = sg.t0; t < sg.t1 && ok; ++t, ++it) {
         const int b = it & 1;
         ok = mbar_wait(bar(B_S_FULL + b), (it >> 1) & 1, s_abort);
         if (!ok) break;
         tc_fence_after();
+        float s[kTileTok];
+        tmem_ld128(t_lane + b * 128, s);
         const int vis = min(kTileTok, max(0, pos + 1 - t * kTileTok));   // visible columns of this row
-        const uint32_t s_addr = t_lane + b * 128;
-        // pass 1: row maximum over the visible columns
         float mx = -INFINITY;
+        if (live) {
+          if (vis >= kTileTok) {
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          float s[32];
-          tmem_ld32(s_addr + ch * 32, s);
-          if (live) {
+            for (int x = 0; x < kTileTok; ++x) mx = fmaxf(mx, s[x]);
+          } else {
 #pragma unroll
-            for (int x = 0; x < 32; ++x) mx = (ch * 32 + x < vis) ? fmaxf(mx, s[x]) : mx;
+            for (int x = 0; x < kTileTok; ++x) mx = (x < vis) ? fmaxf(mx, s[x]) : mx;
           }
         }
-        const float m_new = fmaxf(m_run, mx * scale_log2);
-        const float m_safe = (m_new == -INFINITY) ? 0.0f : m_new;
-        const float alpha = ex2(m_run - m_safe);
-        // the previous use of this P buffer (tile it - 2) was consumed by an MMA
-        // whose completion this thread already saw (o_full of it - 2)
+        mx *= scale_log2;
+        float factor = 1.0f;
+        bool need = false;
+        if (t == sg.t0) {
+          m_ref = mx;                                   // the run's first P.V starts a fresh O
+        } else if (mx > m_ref + 8.0f) {
+          factor = ex2(m_ref - mx);
+          m_ref = mx;
+          l_run *= factor;
+          need = true;
+        }
+        if (__any_sync(0xffffffffu, need)) {
+          // rescale this warp's O rows in TMEM before the next P.V accumulates
+          ok = wait_pv(it - 1);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            float o[32];
+            tmem_ld32(o_addr + ch * 32, o);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) o[x] *= factor;
+            tmem_st32(o_addr + ch * 32, o);
+          }
+          tmem_st_wait();
+        }
+        const float m_safe = (m_ref == -INFINITY) ? 0.0f : m_ref;
+        // P[b] was last read by the P.V of tile it - 2
+        if (it >= 2) { ok = wait_pv(it - 2); if (!ok) break; }
         const uint32_t p_row = base + kOffP + b * kPBytes + row * 128;
         float psum = 0.0f;
-        // pass 2: p = exp2(s * scale - m), bf16, swizzled store
+        if (live) {
+          const bool full = vis >= kTileTok;
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          float s[32];
-          tmem_ld32(s_addr + ch * 32, s);
-          if (live) {
-            uint32_t pk[16];
+          for (int chunk = 0; chunk < kTileTok / 8; ++chunk) {        // 8 tokens = one 16-byte chunk
+            float p[8];
 #pragma unroll
-            for (int x = 0; x < 32; x += 2) {
-              const int col = ch * 32 + x;
-              float p0 = ex2(fmaf(s[x], scale_log2, -m_safe));
-              float p1 = ex2(fmaf(s[x + 1], scale_log2, -m_safe));
-              p0 = (col < vis) ? p0 : 0.0f;
-              p1 = (col + 1 < vis) ? p1 : 0.0f;
-              psum += p0 + p1;
-              pk[x >> 1] = pack_bf16(p0, p1);
+            for (int x = 0; x < 8; ++x) {
+              const float e = ex2(fmaf(s[chunk * 8 + x], scale_log2, -m_safe));
+              p[x] = (full || chunk * 8 + x < vis) ? e : 0.0f;
+              psum += p[x];
             }
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-              const int chunk = ch * 4 + q4;                       // 16-byte chunk = 8 tokens
-              const uint32_t addr = p_row + (chunk >> 3) * (kTcRows * 128) +
-                                    (((chunk & 7) ^ (row & 7)) << 4);
-              st_shared_v4(addr, pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
-            }
+            const uint32_t addr = p_row + (chunk >> 3) * (kTcRows * 128) +
+                                  (((chunk & 7) ^ (row & 7)) << 4);
+            st_shared_v4(addr, pack_bf16(p[0], p[1]), pack_bf16(p[2], p[3]), pack_bf16(p[4], p[5]),
+                         pack_bf16(p[6], p[7]));
           }
         }
-        if (live) { l_run = l_run * alpha + psum; m_run = m_new; }
+        l_run += psum;
         // last tile of the pair: V rows at or beyond the request's key count
         // must be finite (0 x NaN would poison the row): zero them once the
         // copy has landed
@@ -539,12 +570,15 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         tc_fence_before();
         fence_async_smem();
         mbar_arrive(bar(B_P_FULL + b));
-        if (t > sg.t0) ok = fold_o(it - 1);
-        alpha_pending = alpha;
       }
       if (!ok) break;
-      ok = fold_o(it - 1);                              // drain the last tile of the run
+      ok = wait_pv(it - 1);                            // the run's last P.V
       if (!ok) break;
+      tc_fence_after();
+      float acc[kD];
+      tmem_ld128(o_addr, acc);
+      tc_fence_before();
+      float m_run = m_ref;
 
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.n_tiles);
       bool write_rows = whole;
