@@ -7,7 +7,9 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libdscale.so")
+# DSCALE_LIB points the binding at another build of the same library (for
+# example one compiled with -DDSCALE_TRACE); the default is the in-tree build.
+_LIB_PATH = os.environ.get("DSCALE_LIB") or os.path.join(_HERE, "libdscale.so")
 
 if not os.path.exists(_LIB_PATH):
     raise ImportError(

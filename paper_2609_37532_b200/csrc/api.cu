@@ -246,7 +246,7 @@ const int32_t* dscale_ws_field(const void* ws, int n_bs, int field) {
 int dscale_launches_per_call(int which) {
   switch (which) {
     case 0: return 1;   // dvl_alloc_kernel
-    case 1: return 1;   // attn_tc_kernel (split-KV merge happens inside it)
+    case 1: return 1;   // attn_tc_kernel (cut pairs are merged inside it)
     case 2: return 1;   // accept_kernel
     case 3: return 1;   // attn_simt_kernel
     default: return 0;

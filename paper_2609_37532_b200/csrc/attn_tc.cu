@@ -12,9 +12,10 @@
 // list (the per-request tile prefix comes from the allocation kernel); CTA c
 // of a persistent grid of one CTA per SM takes the contiguous slice
 // [c T / C, (c+1) T / C).  A slice cuts at most its first and its last pair;
-// those write an un-normalised partial (O, m, l) to the workspace, and the
-// last CTA to arrive at a pair (a ticket counter, nobody waits) merges the
-// partials and writes the rows.  Pairs inside a slice are written directly.
+// those write an un-normalised partial (O, m, l) to the workspace; after its
+// main loop a CTA publishes its partials (fence + a ticket per pair) and the
+// last CTA to reach a pair merges it and writes its rows -- nobody waits for
+// another CTA.  Pairs inside a slice are written directly.
 // The grid and every address are independent of the lengths, so a captured
 // launch replays at any mix of lengths.
 //
@@ -221,6 +222,15 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
                "r"(d) : "memory");
 }
 
+#ifdef DSCALE_TRACE
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t;
+}
+#define TRACE(slot) do { if (tid == 0 && (slot) < 64) trace[(slot)] = gtime(); } while (0)
+#else
+#define TRACE(slot) do { } while (0)
+#endif
+
 // ------------------------------------------------------------------ schedule
 // One maximal run of tiles of a single (request, kv-head) pair inside a CTA's slice.
 struct Segment {
@@ -272,13 +282,16 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   unsigned char* sm = smem_dyn + (base - raw);
   volatile int* s_abort = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm + kOffMisc);
-  int* s_ticket = reinterpret_cast<int*>(sm + kOffMisc + 8);
-  volatile int* s_dummy = reinterpret_cast<volatile int*>(sm + kOffMisc + 12);
+  int* s_ticket = reinterpret_cast<int*>(sm + kOffMisc + 8);          // two ints
+  volatile int* s_dummy = reinterpret_cast<volatile int*>(sm + kOffMisc + 16);
   int* s_tile = reinterpret_cast<int*>(sm + kOffTile);
   auto bar = [&](int b) { return base + kOffBar + 8u * b; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int c = blockIdx.x;
+#ifdef DSCALE_TRACE
+  const unsigned long long t_entry = gtime();
+#endif
   int* hdr = ws_ptr<int>(a.ws, L.hdr);
   const int n_bs = a.n_bs, n_kv = a.n_kv_heads, Hq = a.n_q_heads;
 
@@ -454,22 +467,19 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
     float* part_o = ws_ptr<float>(a.ws, L.part_o);
     float* part_ml = ws_ptr<float>(a.ws, L.part_ml);
-    int* pair_cnt = ws_ptr<int>(a.ws, L.pair_cnt);
     __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a.out);
+    int* pair_cnt = ws_ptr<int>(a.ws, L.pair_cnt);
 
     Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
     Segment sg;
     unsigned it = 0;
     bool ok = true;
-    // bounded barrier among the 128 softmax threads (an mbarrier, so that a
-    // thread that gave up cannot leave the others stuck)
-    unsigned group_phase = 0;
-    auto group_sync = [&]() -> bool {
-      mbar_arrive(bar(B_GROUP));
-      const bool r = mbar_wait(bar(B_GROUP), group_phase & 1, s_abort);
-      ++group_phase;
-      return r;
-    };
+#ifdef DSCALE_TRACE
+    unsigned long long* trace = ws_ptr<unsigned long long>(a.ws, L.trace) + (size_t)c * 64;
+    int tr = 2;
+    if (tid == 0) { for (int x = 0; x < 64; ++x) trace[x] = 0; trace[0] = t_entry; trace[1] = gtime(); }
+#endif
+    int pend_i[2], pend_g[2], pend_n[2], n_pend = 0;   // partial runs: at most the slice's first and last
     auto wait_pv = [&](unsigned pt) -> bool {        // P.V of tile pt has completed
       return mbar_wait(bar(B_O_FULL + (pt & 1)), (pt >> 1) & 1, s_abort);
     };
@@ -489,6 +499,9 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         ok = mbar_wait(bar(B_S_FULL + b), (it >> 1) & 1, s_abort);
         if (!ok) break;
         tc_fence_after();
+#ifdef DSCALE_TRACE
+        if (t == sg.t0) { TRACE(tr); ++tr; }
+#endif
         float s[kTileTok];
         tmem_ld128(t_lane + b * 128, s);
         const int vis = min(kTileTok, max(0, pos + 1 - t * kTileTok));   // visible columns of this row
@@ -572,78 +585,141 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         mbar_arrive(bar(B_P_FULL + b));
       }
       if (!ok) break;
+#ifdef DSCALE_TRACE
+      TRACE(tr); ++tr;
+#endif
       ok = wait_pv(it - 1);                            // the run's last P.V
       if (!ok) break;
+#ifdef DSCALE_TRACE
+      TRACE(tr); ++tr;
+#endif
       tc_fence_after();
       float acc[kD];
       tmem_ld128(o_addr, acc);
       tc_fence_before();
-      float m_run = m_ref;
 
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.n_tiles);
-      bool write_rows = whole;
-      if (!whole) {
-        // un-normalised partial to the workspace, then the pair's ticket
+      if (whole) {
+        if (live) {
+          const float inv = 1.0f / l_run;
+          uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(oi + j_row) * Hq + sg.g * 4 + h_loc) * kD);
+#pragma unroll
+          for (int d = 0; d < kD; d += 8) {
+            dst[d >> 3] = make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv),
+                                     pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
+                                     pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv),
+                                     pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
+          }
+        }
+      } else {
+        // A run that covers only part of its pair: store the un-normalised partial
+        // and go on.  Nothing in the main loop waits on global memory (a round trip
+        // costs microseconds while every SM is streaming); the partial is
+        // published after the loop.
         const int slot_id = c * 2 + (sg.first_of_cta ? 0 : 1);
         if (live) {
           float4* po = reinterpret_cast<float4*>(part_o + ((size_t)slot_id * kTcRows + row) * kD);
 #pragma unroll
           for (int d = 0; d < kD; d += 4) po[d >> 2] = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
-          part_ml[((size_t)slot_id * kTcRows + row) * 2] = m_run;
-          part_ml[((size_t)slot_id * kTcRows + row) * 2 + 1] = l_run;
+          *reinterpret_cast<float2*>(&part_ml[((size_t)slot_id * kTcRows + row) * 2]) =
+              make_float2(m_ref, l_run);
         }
+        pend_i[n_pend] = sg.i; pend_g[n_pend] = sg.g; pend_n[n_pend] = sg.n_tiles;
+        ++n_pend;
+      }
+#ifdef DSCALE_TRACE
+      TRACE(tr); ++tr;
+#endif
+    }
+#ifdef DSCALE_TRACE
+    TRACE(60);
+#endif
+    // ---- publish this CTA's partial runs; merge the pairs it is the last to reach.
+    // One fence, one ticket per pair (taken by two different threads at once),
+    // then one round trip to L2 per pair: nobody ever waits for another CTA.
+    if (ok && n_pend > 0) {
+      unsigned group_phase = 0;
+      auto group_sync = [&]() -> bool {                 // bounded barrier of the 128 softmax threads
+        mbar_arrive(bar(B_GROUP));
+        const bool r = mbar_wait(bar(B_GROUP), group_phase & 1, s_abort);
+        ++group_phase;
+        return r;
+      };
+      __threadfence();
+      ok = group_sync();
+      if (ok && lane == 0 && warp < n_pend) {
+        const int x = warp;
+        const long long p0 = ((long long)s_tile[pend_i[x]] * n_kv) + (long long)pend_g[x] * pend_n[x];
+        const int n_contrib = cta_of(p0 + pend_n[x] - 1, T, C) - cta_of(p0, T, C) + 1;
+        int* cnt = &pair_cnt[pend_i[x] * n_kv + pend_g[x]];
+        const int old = atomicAdd(cnt, 1);
+        s_ticket[x] = (old == n_contrib - 1);
+        if (old == n_contrib - 1) *cnt = 0;             // ready for the next launch
+      }
+      if (ok) ok = group_sync();
+      for (int x = 0; ok && x < n_pend; ++x) {
+        if (!s_ticket[x]) continue;
         __threadfence();
-        if (!group_sync()) { ok = false; break; }
-        const long long p0 = ((long long)s_tile[sg.i] * n_kv) + (long long)sg.g * sg.n_tiles;
-        const int c_lo = cta_of(p0, T, C), c_hi = cta_of(p0 + sg.n_tiles - 1, T, C);
-        if (tid == 0) {
-          const int old = atomicAdd(&pair_cnt[sg.i * n_kv + sg.g], 1);
-          *s_ticket = (old == c_hi - c_lo);
-          if (old == c_hi - c_lo) pair_cnt[sg.i * n_kv + sg.g] = 0;   // ready for the next launch
-        }
-        if (!group_sync()) { ok = false; break; }
-        if (*s_ticket) {
-          __threadfence();
-          write_rows = true;
-          if (live) {
-            for (int cc = c_lo; cc <= c_hi; ++cc) {
-              if (cc == c) continue;
-              const int sid = cc * 2 + (slice_begin(cc, T, C) >= p0 ? 0 : 1);
-              const float m_o = __ldcg(&part_ml[((size_t)sid * kTcRows + row) * 2]);
-              const float l_o = __ldcg(&part_ml[((size_t)sid * kTcRows + row) * 2 + 1]);
-              const float m_tot = fmaxf(m_run, m_o);
-              const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
-              const float w_me = ex2(m_run - m_s), w_o = ex2(m_o - m_s);
-              const float4* po = reinterpret_cast<const float4*>(part_o + ((size_t)sid * kTcRows + row) * kD);
+        const int pi = pend_i[x], pg = pend_g[x];
+        const int ki = ws_ptr<int>(a.ws, L.k)[pi];
+        const int oi = ws_ptr<int>(a.ws, L.offset)[pi];
+        const long long p0 = ((long long)s_tile[pi] * n_kv) + (long long)pg * pend_n[x];
+        const int c_lo = cta_of(p0, T, C), c_hi = cta_of(p0 + pend_n[x] - 1, T, C);
+        // warp w owns tile rows w, w + 4, ...; lane l owns columns 4 l .. 4 l + 3, so
+        // partial loads and output stores are contiguous; two contributors per trip
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {                  // 8 tile rows per pass
+        float4 av[8];
+        float mr[8], lr[8];
 #pragma unroll
-              for (int d = 0; d < kD; d += 4) {
-                const float4 v = __ldcg(&po[d >> 2]);
-                acc[d] = acc[d] * w_me + v.x * w_o;
-                acc[d + 1] = acc[d + 1] * w_me + v.y * w_o;
-                acc[d + 2] = acc[d + 2] * w_me + v.z * w_o;
-                acc[d + 3] = acc[d + 3] * w_me + v.w * w_o;
-              }
-              l_run = l_run * w_me + l_o * w_o;
-              m_run = m_tot;
+        for (int r = 0; r < 8; ++r) { av[r] = make_float4(0.f, 0.f, 0.f, 0.f); mr[r] = -INFINITY; lr[r] = 0.f; }
+        for (int cb = c_lo; cb <= c_hi; cb += 2) {
+          float4 v[2][8];
+          float2 ml[2][8];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int cc = min(cb + u, c_hi);
+            const int sid = cc * 2 + (slice_begin(cc, T, C) >= p0 ? 0 : 1);
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+              const int rr = min(warp + 4 * (r + 8 * half), 4 * ki - 1);
+              v[u][r] = __ldcg(reinterpret_cast<const float4*>(part_o + ((size_t)sid * kTcRows + rr) * kD) + lane);
+              ml[u][r] = __ldcg(reinterpret_cast<const float2*>(&part_ml[((size_t)sid * kTcRows + rr) * 2]));
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            if (cb + u > c_hi) break;
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+              const float m_tot = fmaxf(mr[r], ml[u][r].x);
+              const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
+              const float w0 = ex2(mr[r] - m_s), w1 = ex2(ml[u][r].x - m_s);
+              av[r].x = av[r].x * w0 + v[u][r].x * w1; av[r].y = av[r].y * w0 + v[u][r].y * w1;
+              av[r].z = av[r].z * w0 + v[u][r].z * w1; av[r].w = av[r].w * w0 + v[u][r].w * w1;
+              lr[r] = lr[r] * w0 + ml[u][r].y * w1;
+              mr[r] = m_tot;
             }
           }
         }
-        if (!group_sync()) { ok = false; break; }            // s_ticket is reused by the next run
-      }
-      if (write_rows && live) {
-        const float inv = 1.0f / l_run;
-        uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(oi + j_row) * Hq + sg.g * 4 + h_loc) * kD);
 #pragma unroll
-        for (int d = 0; d < kD; d += 8) {
-          dst[d >> 3] = make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv),
-                                   pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
-                                   pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv),
-                                   pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
+        for (int r = 0; r < 8; ++r) {
+          const int rr = warp + 4 * (r + 8 * half);                  // tile row = 4 j + h_local
+          if (rr < 4 * ki) {
+            const float inv = 1.0f / lr[r];
+            uint2 pk = make_uint2(pack_bf16(av[r].x * inv, av[r].y * inv),
+                                  pack_bf16(av[r].z * inv, av[r].w * inv));
+            *reinterpret_cast<uint2*>(out + ((size_t)(oi + (rr >> 2)) * Hq + pg * 4 + (rr & 3)) * kD + lane * 4) = pk;
+          }
+        }
         }
       }
     }
   }
 
+#ifdef DSCALE_TRACE
+  if (tid == 0) ws_ptr<unsigned long long>(a.ws, L.trace)[(size_t)c * 64 + 61] = gtime();
+#endif
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();

@@ -28,7 +28,7 @@ enum HdrWord {
 
 struct WsLayout {
   size_t hdr, k, k0, offset, q_start, q_end, tokens, positions, kv_refs, row_req, top1,
-      kv_len, tile_prefix, qscores, amax_val, amax_idx, pair_cnt, part_o, part_ml, total;
+      kv_len, tile_prefix, qscores, amax_val, amax_idx, pair_cnt, part_o, part_ml, trace, total;
 };
 
 __host__ __device__ inline size_t ws_align(size_t x) { return (x + 255) & ~size_t(255); }
@@ -59,6 +59,8 @@ __host__ __device__ inline WsLayout ws_layout(int n_bs, int n_kv_heads, int num_
   // (128 fp32 accumulators) plus (row max, row sum)
   L.part_o = o;      o = ws_align(o + size_t(num_ctas) * 2 * kTcRows * kD * 4);
   L.part_ml = o;     o = ws_align(o + size_t(num_ctas) * 2 * kTcRows * 2 * 4);
+  // per-CTA timestamps, written only by builds with -DDSCALE_TRACE
+  L.trace = o;       o = ws_align(o + size_t(num_ctas) * 64 * 8);
   L.total = o;
   return L;
 }
