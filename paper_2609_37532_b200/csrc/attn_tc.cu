@@ -12,14 +12,18 @@
 // list (the per-request tile prefix comes from the allocation kernel); CTA c
 // of a persistent grid of one CTA per SM takes the contiguous slice
 // [c T / C, (c+1) T / C).  A slice cuts at most its first and its last pair;
-// those write an un-normalised partial (O, m, l) to the workspace; after its
-// main loop a CTA publishes its partials (fence + a ticket per pair) and the
-// last CTA to reach a pair merges it and writes its rows -- nobody waits for
-// another CTA.  Pairs inside a slice are written directly.
+// those produce an un-normalised partial (O, m, l).  Partials are published with
+// a fence and a ticket on a per-pair counter, and the last CTA to reach a pair
+// merges it and writes its rows -- nobody waits for another CTA.  The partial of
+// a slice's first run is published in the background by a helper warp; the CTA
+// that ends its slice inside a pair normally finds the other partials already
+// published, has them copied into shared memory behind its last tiles and
+// finishes the pair without a global round trip.  Pairs inside a slice are
+// written directly.
 // The grid and every address are independent of the lengths, so a captured
 // launch replays at any mix of lengths.
 //
-// Pipeline inside a CTA (192 threads):
+// Pipeline inside a CTA (224 threads):
 //   warp 4     producer: per tile, 16 + 16 TMA box copies (one 16-token page
 //              x 64 columns each, 128-byte swizzle) of K then V into a 5-deep
 //              ring of 32 KB slots; page ids are fetched one tile ahead.
@@ -32,6 +36,7 @@
 //              TMEM for a whole run of tiles (the second MMA accumulates onto
 //              it); it is only rescaled in place when a row maximum outgrows its
 //              reference by 2^8, and read back once per run for the epilogue.
+//   warp 6     publisher: fence + ticket for the first run's partial.
 // S is double-buffered in TMEM (2 x 128 columns) next to O (128 columns), P and
 // Q are double-buffered in shared memory, so the MMA of tile t+1 overlaps the
 // softmax of tile t.
@@ -50,7 +55,7 @@ namespace dscale {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr int kSoftmaxThreads = 128;
 constexpr int kStages = 5;
 constexpr int kSlotBytes = kTileTok * kD * 2;           // 32 KB: one K or V tile
@@ -65,17 +70,21 @@ constexpr int kOffQ = 0;                                 // 2 x 16 KB
 constexpr int kOffP = kOffQ + 2 * kQBytes;               // 2 x 16 KB
 constexpr int kOffKV = kOffP + 2 * kPBytes;              // 5 x 32 KB
 constexpr int kOffBar = kOffKV + kStages * kSlotBytes;   // mbarriers
-constexpr int kNumBars = 2 * kStages + 2 + 2 + 2 + 2 + 2 + 1;
-constexpr int kOffMisc = kOffBar + 8 * 24;               // tmem base, abort flag, ticket
-constexpr int kOffTile = kOffMisc + 32;                  // tile prefix, kMaxNbs + 1 ints
+constexpr int kNumBars = 2 * kStages + 2 + 2 + 2 + 2 + 2 + 5;
+constexpr int kOffMisc = kOffBar + 8 * 32;               // tmem base, abort flag, tickets
+constexpr int kOffTile = kOffMisc + 48;                  // tile prefix, kMaxNbs + 1 ints
 constexpr int kSmemUse = kOffTile + (kMaxNbs + 1) * 4 + 12;
 constexpr int kSmemBytes = kSmemUse + 1024;              // slack for base alignment
-static_assert(kNumBars <= 24, "barrier area");
+static_assert(kNumBars <= 32, "barrier area");
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
 
 enum Bar { B_KV_FULL = 0, B_KV_EMPTY = kStages, B_Q_FULL = 2 * kStages, B_Q_EMPTY = B_Q_FULL + 2,
            B_S_FULL = B_Q_EMPTY + 2, B_P_FULL = B_S_FULL + 2, B_O_FULL = B_P_FULL + 2,
-           B_GROUP = B_O_FULL + 2 };
+           B_GROUP = B_O_FULL + 2,   // the 128 softmax threads among themselves
+           B_PART = B_GROUP + 1,     // softmax -> publisher: the first run's partial is stored
+           B_PUB = B_PART + 1,       // publisher -> softmax: that partial is published
+           B_PARTNER = B_PUB + 1,    // producer -> softmax: partner partials landed (or not)
+           B_MERGE = B_PARTNER + 1 };// bulk copies of the end-phase merge
 
 // ------------------------------------------------------------------ PTX glue
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -112,6 +121,36 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (*abort_flag) return false;
     if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
   }
+}
+__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+// plain (untiled) bulk copy global -> shared, completion on an mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_async_all() {
+  asm volatile("fence.proxy.async;" ::: "memory");
+}
+__device__ __forceinline__ float4 ld_shared_v4f(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 ld_shared_v2f(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
 }
 __device__ __forceinline__ void fence_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -264,7 +303,24 @@ struct Scheduler {
     pos += s.t1 - s.t0;
     return true;
   }
+  __device__ bool more() const { return pos < end; }   // runs left after the one just returned
 };
+
+// How a run's result reaches the output.
+//   WHOLE    the run is its whole pair: rows are written directly.
+//   PUBLISH  first run of a slice, more runs follow: the partial is stored and a
+//            publisher warp publishes it in the background.
+//   TAIL     last run of a slice, the pair starts in this slice: the producer
+//            checks whether all other contributors are published and, if so,
+//            copies their partials into shared memory (fast path).
+//   FINAL    last run, any other shape: stored and published after the main loop.
+enum RunKind { RUN_WHOLE = 0, RUN_PUBLISH = 1, RUN_TAIL = 2, RUN_FINAL = 3 };
+__device__ __forceinline__ int run_kind(const Segment& s, bool more) {
+  if (s.t0 == 0 && s.t1 == s.n_tiles) return RUN_WHOLE;
+  if (more) return RUN_PUBLISH;                 // only a slice's first run can be partial and not last
+  return (s.t0 == 0) ? RUN_TAIL : RUN_FINAL;
+}
+constexpr int kMaxFastPartners = 3;
 
 __device__ __forceinline__ long long slice_begin(int c, long long T, int C) { return (long long)c * T / C; }
 // the CTA whose slice holds linear tile index L
@@ -283,6 +339,8 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   volatile int* s_abort = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm + kOffMisc);
   int* s_ticket = reinterpret_cast<int*>(sm + kOffMisc + 8);          // two ints
+  volatile int* s_fast = reinterpret_cast<volatile int*>(sm + kOffMisc + 20);      // partner partials in smem
+  volatile int* s_head_last = reinterpret_cast<volatile int*>(sm + kOffMisc + 24); // publisher took the last ticket
   volatile int* s_dummy = reinterpret_cast<volatile int*>(sm + kOffMisc + 16);
   int* s_tile = reinterpret_cast<int*>(sm + kOffTile);
   auto bar = [&](int b) { return base + kOffBar + 8u * b; };
@@ -303,6 +361,10 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       mbar_init(bar(B_O_FULL + b), 1);
     }
     mbar_init(bar(B_GROUP), kSoftmaxThreads);
+    mbar_init(bar(B_PART), kSoftmaxThreads);
+    mbar_init(bar(B_PUB), 1);
+    mbar_init(bar(B_PARTNER), 1);
+    mbar_init(bar(B_MERGE), 1);
     *s_abort = 0;
     *s_dummy = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -381,6 +443,42 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           }
         }
       }
+      if (ok && run_kind(sg, sch.more()) == RUN_TAIL) {
+        // The slice ends inside this pair.  If every other contributor has already
+        // published its partial (the usual case: they computed theirs at the start
+        // of their slices), fetch those partials into ring slots behind the last
+        // tiles, so that the softmax warps can finish the pair without a single
+        // global round trip.
+        const long long p0 = ((long long)s_tile[sg.i] * n_kv) + (long long)sg.g * sg.n_tiles;
+        const int c_hi = cta_of(p0 + sg.n_tiles - 1, T, C);
+        const int others = c_hi - c;                       // this CTA holds the pair's first tiles
+        int fast = 0;
+        if (others <= kMaxFastPartners) {
+          const int seen = ld_acquire_gpu(&ws_ptr<int>(a.ws, L.pair_cnt)[sg.i * n_kv + sg.g]);
+          if (seen == others) fast = others;
+        }
+        if (fast) {
+          fence_async_all();
+          const float* part_o = ws_ptr<float>(a.ws, L.part_o);
+          const float* part_ml = ws_ptr<float>(a.ws, L.part_ml);
+          float* s_ml = reinterpret_cast<float*>(sm + kOffQ + ((seg + 1) & 1) * kQBytes);  // unused Q buffer
+          for (int x = 0; x < fast && ok; ++x, ++u) {
+            const int sid = (c + 1 + x) * 2;               // their run starts their slice: slot 0
+            const int slot = u % kStages;
+            ok = mbar_wait(bar(B_KV_EMPTY + slot), ((u / kStages) & 1) ^ 1, s_abort);
+            if (!ok) break;
+            if (lane == 0) {
+              mbar_expect_tx_only(bar(B_PARTNER), kTcRows * kD * 4);
+              bulk_load(base + kOffKV + slot * kSlotBytes, part_o + (size_t)sid * kTcRows * kD,
+                        kTcRows * kD * 4, bar(B_PARTNER));
+            }
+            reinterpret_cast<float4*>(s_ml + x * kTcRows * 2)[lane] =
+                __ldcg(reinterpret_cast<const float4*>(part_ml + (size_t)sid * kTcRows * 2) + lane);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) { *s_fast = ok ? fast : 0; mbar_arrive(bar(B_PARTNER)); }
+      }
       ++seg;
     }
     // on an aborted run, let the copies already issued land before the CTA's
@@ -448,6 +546,29 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       if (ok && it >= 1) ok = issue_pv(it - 1);
     }
     __syncwarp();
+  } else if (warp == 6) {
+    // ========================================================= publisher warp
+    // Publishes the partial of the slice's first run in the background: waits
+    // until the softmax threads have stored it, fences, and takes a ticket on the
+    // pair's counter.  The fence and the atomic are global round trips of a few
+    // microseconds while the SM streams; here they delay nobody.
+    Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
+    Segment sg;
+    if (sch.next(sg) && run_kind(sg, sch.more()) == RUN_PUBLISH) {
+      if (mbar_wait(bar(B_PART), 0, s_abort)) {
+        __threadfence();
+        if (lane == 0) {
+          const long long p0 = ((long long)s_tile[sg.i] * n_kv) + (long long)sg.g * sg.n_tiles;
+          const int n_contrib = cta_of(p0 + sg.n_tiles - 1, T, C) - cta_of(p0, T, C) + 1;
+          int* cnt = &ws_ptr<int>(a.ws, L.pair_cnt)[sg.i * n_kv + sg.g];
+          const int old = atomicAdd(cnt, 1);
+          *s_head_last = (old == n_contrib - 1);          // then this CTA merges it after its loop
+          if (old == n_contrib - 1) *cnt = 0;             // ready for the next launch
+          mbar_arrive(bar(B_PUB));
+        }
+      }
+    }
+    __syncwarp();
   } else {
     // ====================================================== softmax warps 0-3
     // rows of capacity beyond M_live are written as zero, spread over the grid
@@ -479,7 +600,9 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     int tr = 2;
     if (tid == 0) { for (int x = 0; x < 64; ++x) trace[x] = 0; trace[0] = t_entry; trace[1] = gtime(); }
 #endif
-    int pend_i[2], pend_g[2], pend_n[2], n_pend = 0;   // partial runs: at most the slice's first and last
+    int head_i = -1, head_g = 0, head_n = 0;   // first run, published in the background
+    int fin_i = -1, fin_g = 0, fin_n = 0;      // last run, published after the loop
+    int seg = 0;
     auto wait_pv = [&](unsigned pt) -> bool {        // P.V of tile pt has completed
       return mbar_wait(bar(B_O_FULL + (pt & 1)), (pt >> 1) & 1, s_abort);
     };
@@ -598,24 +721,57 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       tmem_ld128(o_addr, acc);
       tc_fence_before();
 
-      const bool whole = (sg.t0 == 0 && sg.t1 == sg.n_tiles);
-      if (whole) {
-        if (live) {
-          const float inv = 1.0f / l_run;
-          uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(oi + j_row) * Hq + sg.g * 4 + h_loc) * kD);
+      const int kind = run_kind(sg, sch.more());
+      bool write_rows = (kind == RUN_WHOLE);
+      bool store_partial = (kind == RUN_PUBLISH || kind == RUN_FINAL);
+      if (kind == RUN_TAIL) {
+        ok = mbar_wait(bar(B_PARTNER), 0, s_abort);
+        if (!ok) break;
+        const int fast = *s_fast;
+        if (fast > 0) {
+          // all other contributors' partials sit in ring slots 2 it, 2 it + 1, ...:
+          // fold them into this thread's row and finish the pair here
+          if (live) {
+            const uint32_t ml_base = base + kOffQ + ((seg + 1) & 1) * kQBytes;
+            for (int x = 0; x < fast; ++x) {
+              const uint32_t o_row = base + kOffKV + ((2 * it + x) % kStages) * kSlotBytes + row * (kD * 4);
+              const float2 ml = ld_shared_v2f(ml_base + (x * kTcRows + row) * 8);
+              const float m_tot = fmaxf(m_ref, ml.x);
+              const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
+              const float w_me = ex2(m_ref - m_s), w_o = ex2(ml.x - m_s);
 #pragma unroll
-          for (int d = 0; d < kD; d += 8) {
-            dst[d >> 3] = make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv),
-                                     pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
-                                     pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv),
-                                     pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
+              for (int d = 0; d < kD; d += 4) {
+                const float4 v = ld_shared_v4f(o_row + d * 4);
+                acc[d] = acc[d] * w_me + v.x * w_o;
+                acc[d + 1] = acc[d + 1] * w_me + v.y * w_o;
+                acc[d + 2] = acc[d + 2] * w_me + v.z * w_o;
+                acc[d + 3] = acc[d + 3] * w_me + v.w * w_o;
+              }
+              l_run = l_run * w_me + ml.y * w_o;
+              m_ref = m_tot;
+            }
           }
+          if (tid == 0) pair_cnt[sg.i * n_kv + sg.g] = 0;      // ready for the next launch
+          write_rows = true;
+        } else {
+          store_partial = true;                                // ordinary path after the loop
         }
-      } else {
-        // A run that covers only part of its pair: store the un-normalised partial
-        // and go on.  Nothing in the main loop waits on global memory (a round trip
-        // costs microseconds while every SM is streaming); the partial is
-        // published after the loop.
+      }
+      if (write_rows && live) {
+        const float inv = 1.0f / l_run;
+        uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(oi + j_row) * Hq + sg.g * 4 + h_loc) * kD);
+#pragma unroll
+        for (int d = 0; d < kD; d += 8) {
+          dst[d >> 3] = make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv),
+                                   pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
+                                   pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv),
+                                   pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
+        }
+      }
+      if (store_partial) {
+        // A run that covers only part of its pair: store the un-normalised partial.
+        // Nothing in the main loop waits on global memory (a round trip costs
+        // microseconds while every SM is streaming).
         const int slot_id = c * 2 + (sg.first_of_cta ? 0 : 1);
         if (live) {
           float4* po = reinterpret_cast<float4*>(part_o + ((size_t)slot_id * kTcRows + row) * kD);
@@ -624,9 +780,14 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           *reinterpret_cast<float2*>(&part_ml[((size_t)slot_id * kTcRows + row) * 2]) =
               make_float2(m_ref, l_run);
         }
-        pend_i[n_pend] = sg.i; pend_g[n_pend] = sg.g; pend_n[n_pend] = sg.n_tiles;
-        ++n_pend;
+        if (kind == RUN_PUBLISH) {
+          mbar_arrive(bar(B_PART));                            // the publisher warp takes over
+          head_i = sg.i; head_g = sg.g; head_n = sg.n_tiles;
+        } else {
+          fin_i = sg.i; fin_g = sg.g; fin_n = sg.n_tiles;      // published below, after the loop
+        }
       }
+      ++seg;
 #ifdef DSCALE_TRACE
       TRACE(tr); ++tr;
 #endif
@@ -634,84 +795,105 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 #ifdef DSCALE_TRACE
     TRACE(60);
 #endif
-    // ---- publish this CTA's partial runs; merge the pairs it is the last to reach.
-    // One fence, one ticket per pair (taken by two different threads at once),
-    // then one round trip to L2 per pair: nobody ever waits for another CTA.
-    if (ok && n_pend > 0) {
-      unsigned group_phase = 0;
+    // ---- end phase: publish what is left, merge the pairs this CTA is last to reach
+    if (ok && (fin_i >= 0 || head_i >= 0)) {
+      unsigned group_phase = 0, merge_phase = 0;
       auto group_sync = [&]() -> bool {                 // bounded barrier of the 128 softmax threads
         mbar_arrive(bar(B_GROUP));
         const bool r = mbar_wait(bar(B_GROUP), group_phase & 1, s_abort);
         ++group_phase;
         return r;
       };
-      __threadfence();
-      ok = group_sync();
-      if (ok && lane == 0 && warp < n_pend) {
-        const int x = warp;
-        const long long p0 = ((long long)s_tile[pend_i[x]] * n_kv) + (long long)pend_g[x] * pend_n[x];
-        const int n_contrib = cta_of(p0 + pend_n[x] - 1, T, C) - cta_of(p0, T, C) + 1;
-        int* cnt = &pair_cnt[pend_i[x] * n_kv + pend_g[x]];
-        const int old = atomicAdd(cnt, 1);
-        s_ticket[x] = (old == n_contrib - 1);
-        if (old == n_contrib - 1) *cnt = 0;             // ready for the next launch
-      }
-      if (ok) ok = group_sync();
-      for (int x = 0; ok && x < n_pend; ++x) {
-        if (!s_ticket[x]) continue;
+      int merge_i[2], merge_g[2], merge_n[2], n_merge = 0;
+      if (fin_i >= 0) {
         __threadfence();
-        const int pi = pend_i[x], pg = pend_g[x];
+        ok = group_sync();
+        if (ok && tid == 0) {
+          const long long p0 = ((long long)s_tile[fin_i] * n_kv) + (long long)fin_g * fin_n;
+          const int n_contrib = cta_of(p0 + fin_n - 1, T, C) - cta_of(p0, T, C) + 1;
+          int* cnt = &pair_cnt[fin_i * n_kv + fin_g];
+          const int old = atomicAdd(cnt, 1);
+          s_ticket[0] = (old == n_contrib - 1);
+          if (old == n_contrib - 1) *cnt = 0;           // ready for the next launch
+        }
+        if (ok) ok = group_sync();
+        if (ok && s_ticket[0]) { merge_i[n_merge] = fin_i; merge_g[n_merge] = fin_g; merge_n[n_merge] = fin_n; ++n_merge; }
+      }
+      if (ok && head_i >= 0) {
+        ok = mbar_wait(bar(B_PUB), 0, s_abort);
+        if (ok && *s_head_last) { merge_i[n_merge] = head_i; merge_g[n_merge] = head_g; merge_n[n_merge] = head_n; ++n_merge; }
+      }
+      // Merge: all contributors' partials are bulk-copied into the (now idle) K/V
+      // ring, up to kStages at a time, and each thread combines its own row.
+      for (int x = 0; ok && x < n_merge; ++x) {
+        __threadfence();
+        const int pi = merge_i[x], pg = merge_g[x];
         const int ki = ws_ptr<int>(a.ws, L.k)[pi];
         const int oi = ws_ptr<int>(a.ws, L.offset)[pi];
-        const long long p0 = ((long long)s_tile[pi] * n_kv) + (long long)pg * pend_n[x];
-        const int c_lo = cta_of(p0, T, C), c_hi = cta_of(p0 + pend_n[x] - 1, T, C);
-        // warp w owns tile rows w, w + 4, ...; lane l owns columns 4 l .. 4 l + 3, so
-        // partial loads and output stores are contiguous; two contributors per trip
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {                  // 8 tile rows per pass
-        float4 av[8];
-        float mr[8], lr[8];
+        const bool live = lane < 16 && j_row < ki;
+        const long long p0 = ((long long)s_tile[pi] * n_kv) + (long long)pg * merge_n[x];
+        const int c_lo = cta_of(p0, T, C), c_hi = cta_of(p0 + merge_n[x] - 1, T, C);
+        float acc[kD];
+        float m_run = -INFINITY, l_run = 0.0f;
 #pragma unroll
-        for (int r = 0; r < 8; ++r) { av[r] = make_float4(0.f, 0.f, 0.f, 0.f); mr[r] = -INFINITY; lr[r] = 0.f; }
-        for (int cb = c_lo; cb <= c_hi; cb += 2) {
-          float4 v[2][8];
-          float2 ml[2][8];
+        for (int d = 0; d < kD; ++d) acc[d] = 0.0f;
+        for (int cb = c_lo; cb <= c_hi && ok; cb += kStages) {
+          const int nb = min(kStages, c_hi - cb + 1);
+          ok = group_sync();                            // everybody is done with the ring slots
+          if (!ok) break;
+          if (tid == 0) {
+            fence_async_all();
+            mbar_expect_tx(bar(B_MERGE), nb * kTcRows * kD * 4);
+            for (int y = 0; y < nb; ++y) {
+              const int cc = cb + y;
+              const int sid = cc * 2 + (slice_begin(cc, T, C) >= p0 ? 0 : 1);
+              bulk_load(base + kOffKV + y * kSlotBytes, part_o + (size_t)sid * kTcRows * kD,
+                        kTcRows * kD * 4, bar(B_MERGE));
+            }
+          }
+          float2 ml[kStages];
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int cc = min(cb + u, c_hi);
+          for (int y = 0; y < kStages; ++y) {
+            const int cc = min(cb + y, c_hi);
             const int sid = cc * 2 + (slice_begin(cc, T, C) >= p0 ? 0 : 1);
-#pragma unroll
-            for (int r = 0; r < 8; ++r) {
-              const int rr = min(warp + 4 * (r + 8 * half), 4 * ki - 1);
-              v[u][r] = __ldcg(reinterpret_cast<const float4*>(part_o + ((size_t)sid * kTcRows + rr) * kD) + lane);
-              ml[u][r] = __ldcg(reinterpret_cast<const float2*>(&part_ml[((size_t)sid * kTcRows + rr) * 2]));
-            }
+            ml[y] = live ? __ldcg(reinterpret_cast<const float2*>(&part_ml[((size_t)sid * kTcRows + row) * 2]))
+                         : make_float2(-INFINITY, 0.0f);
           }
+          ok = mbar_wait(bar(B_MERGE), merge_phase & 1, s_abort);
+          ++merge_phase;
+          if (!ok) break;
+          if (live) {
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            if (cb + u > c_hi) break;
+            for (int y = 0; y < kStages; ++y) {
+              if (y < nb) {
+                const uint32_t o_row = base + kOffKV + y * kSlotBytes + row * (kD * 4);
+                const float m_tot = fmaxf(m_run, ml[y].x);
+                const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
+                const float w_me = ex2(m_run - m_s), w_o = ex2(ml[y].x - m_s);
 #pragma unroll
-            for (int r = 0; r < 8; ++r) {
-              const float m_tot = fmaxf(mr[r], ml[u][r].x);
-              const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
-              const float w0 = ex2(mr[r] - m_s), w1 = ex2(ml[u][r].x - m_s);
-              av[r].x = av[r].x * w0 + v[u][r].x * w1; av[r].y = av[r].y * w0 + v[u][r].y * w1;
-              av[r].z = av[r].z * w0 + v[u][r].z * w1; av[r].w = av[r].w * w0 + v[u][r].w * w1;
-              lr[r] = lr[r] * w0 + ml[u][r].y * w1;
-              mr[r] = m_tot;
+                for (int d = 0; d < kD; d += 4) {
+                  const float4 v = ld_shared_v4f(o_row + d * 4);
+                  acc[d] = acc[d] * w_me + v.x * w_o;
+                  acc[d + 1] = acc[d + 1] * w_me + v.y * w_o;
+                  acc[d + 2] = acc[d + 2] * w_me + v.z * w_o;
+                  acc[d + 3] = acc[d + 3] * w_me + v.w * w_o;
+                }
+                l_run = l_run * w_me + ml[y].y * w_o;
+                m_run = m_tot;
+              }
             }
           }
         }
+        if (ok && live) {
+          const float inv = 1.0f / l_run;
+          uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(oi + j_row) * Hq + pg * 4 + h_loc) * kD);
 #pragma unroll
-        for (int r = 0; r < 8; ++r) {
-          const int rr = warp + 4 * (r + 8 * half);                  // tile row = 4 j + h_local
-          if (rr < 4 * ki) {
-            const float inv = 1.0f / lr[r];
-            uint2 pk = make_uint2(pack_bf16(av[r].x * inv, av[r].y * inv),
-                                  pack_bf16(av[r].z * inv, av[r].w * inv));
-            *reinterpret_cast<uint2*>(out + ((size_t)(oi + (rr >> 2)) * Hq + pg * 4 + (rr & 3)) * kD + lane * 4) = pk;
+          for (int d = 0; d < kD; d += 8) {
+            dst[d >> 3] = make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv),
+                                     pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
+                                     pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv),
+                                     pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
           }
-        }
         }
       }
     }
