@@ -443,6 +443,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           }
         }
       }
+#ifndef DSCALE_STREAM_ONLY
       if (ok && run_kind(sg, sch.more()) == RUN_TAIL) {
         // The slice ends inside this pair.  If every other contributor has already
         // published its partial (the usual case: they computed theirs at the start
@@ -479,6 +480,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         __syncwarp();
         if (lane == 0) { *s_fast = ok ? fast : 0; mbar_arrive(bar(B_PARTNER)); }
       }
+#endif
       ++seg;
     }
     // on an aborted run, let the copies already issued land before the CTA's
@@ -489,6 +491,30 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     }
   } else if (warp == 5) {
     // ============================================================ MMA issuer
+#ifdef DSCALE_STREAM_ONLY
+    // probe build: consume every K/V slot as soon as it lands, no math at all;
+    // measures what the TMA page stream alone can sustain
+    if (lane == 0) {
+      Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
+      Segment sg;
+      unsigned u = 0;
+      int seg = 0;
+      bool ok = true;
+      while (ok && sch.next(sg)) {
+        ok = mbar_wait(bar(B_Q_FULL + (seg & 1)), (seg >> 1) & 1, s_abort);
+        for (int t = sg.t0; t < sg.t1 && ok; ++t) {
+          for (int which = 0; which < 2 && ok; ++which, ++u) {
+            ok = mbar_wait(bar(B_KV_FULL + u % kStages), (u / kStages) & 1, s_abort);
+            mbar_arrive(bar(B_KV_EMPTY + u % kStages));
+          }
+        }
+        mbar_arrive(bar(B_Q_EMPTY + (seg & 1)));
+        ++seg;
+      }
+    }
+    __syncwarp();
+  } else if (warp == 7) {
+#endif
     if (lane == 0) {
       Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
       Segment sg;
@@ -554,7 +580,11 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     // microseconds while the SM streams; here they delay nobody.
     Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
     Segment sg;
+#ifdef DSCALE_STREAM_ONLY
+    if (false) {
+#else
     if (sch.next(sg) && run_kind(sg, sch.more()) == RUN_PUBLISH) {
+#endif
       if (mbar_wait(bar(B_PART), 0, s_abort)) {
         __threadfence();
         if (lane == 0) {
@@ -569,7 +599,13 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       }
     }
     __syncwarp();
+#ifdef DSCALE_STREAM_ONLY
+  } else if (warp < 4) {
+    // probe build: no softmax, no output
+  } else if (warp == 8) {
+#else
   } else {
+#endif
     // ====================================================== softmax warps 0-3
     // rows of capacity beyond M_live are written as zero, spread over the grid
     {
@@ -598,6 +634,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 #ifdef DSCALE_TRACE
     unsigned long long* trace = ws_ptr<unsigned long long>(a.ws, L.trace) + (size_t)c * 64;
     int tr = 2;
+    long long wait_cycles = 0, busy_cycles = 0;
     if (tid == 0) { for (int x = 0; x < 64; ++x) trace[x] = 0; trace[0] = t_entry; trace[1] = gtime(); }
 #endif
     int head_i = -1, head_g = 0, head_n = 0;   // first run, published in the background
@@ -619,24 +656,36 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 
       for (int t = sg.t0; t < sg.t1 && ok; ++t, ++it) {
         const int b = it & 1;
+#ifdef DSCALE_TRACE
+        const long long tw0 = clock64();
+#endif
         ok = mbar_wait(bar(B_S_FULL + b), (it >> 1) & 1, s_abort);
         if (!ok) break;
         tc_fence_after();
 #ifdef DSCALE_TRACE
         if (t == sg.t0) { TRACE(tr); ++tr; }
+        const long long tw1 = clock64();
+        wait_cycles += tw1 - tw0;
 #endif
         float s[kTileTok];
         tmem_ld128(t_lane + b * 128, s);
         const int vis = min(kTileTok, max(0, pos + 1 - t * kTileTok));   // visible columns of this row
         float mx = -INFINITY;
         if (live) {
+          // eight independent running maxima: a single chain of 128 dependent
+          // fmax would cost its latency 128 times with one warp per scheduler
+          float m8[8];
+#pragma unroll
+          for (int x = 0; x < 8; ++x) m8[x] = -INFINITY;
           if (vis >= kTileTok) {
 #pragma unroll
-            for (int x = 0; x < kTileTok; ++x) mx = fmaxf(mx, s[x]);
+            for (int x = 0; x < kTileTok; ++x) m8[x & 7] = fmaxf(m8[x & 7], s[x]);
           } else {
 #pragma unroll
-            for (int x = 0; x < kTileTok; ++x) mx = (x < vis) ? fmaxf(mx, s[x]) : mx;
+            for (int x = 0; x < kTileTok; ++x) m8[x & 7] = (x < vis) ? fmaxf(m8[x & 7], s[x]) : m8[x & 7];
           }
+          mx = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])),
+                     fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
         }
         mx *= scale_log2;
         float factor = 1.0f;
@@ -670,21 +719,41 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         const uint32_t p_row = base + kOffP + b * kPBytes + row * 128;
         float psum = 0.0f;
         if (live) {
-          const bool full = vis >= kTileTok;
+          float ps[8];
 #pragma unroll
-          for (int chunk = 0; chunk < kTileTok / 8; ++chunk) {        // 8 tokens = one 16-byte chunk
-            float p[8];
+          for (int x = 0; x < 8; ++x) ps[x] = 0.0f;
+          if (vis >= kTileTok) {
+            // every column visible (all tiles but a pair's last one or two)
 #pragma unroll
-            for (int x = 0; x < 8; ++x) {
-              const float e = ex2(fmaf(s[chunk * 8 + x], scale_log2, -m_safe));
-              p[x] = (full || chunk * 8 + x < vis) ? e : 0.0f;
-              psum += p[x];
+            for (int chunk = 0; chunk < kTileTok / 8; ++chunk) {      // 8 tokens = one 16-byte chunk
+              float p[8];
+#pragma unroll
+              for (int x = 0; x < 8; ++x) {
+                p[x] = ex2(fmaf(s[chunk * 8 + x], scale_log2, -m_safe));
+                ps[x] += p[x];
+              }
+              const uint32_t addr = p_row + (chunk >> 3) * (kTcRows * 128) +
+                                    (((chunk & 7) ^ (row & 7)) << 4);
+              st_shared_v4(addr, pack_bf16(p[0], p[1]), pack_bf16(p[2], p[3]), pack_bf16(p[4], p[5]),
+                           pack_bf16(p[6], p[7]));
             }
-            const uint32_t addr = p_row + (chunk >> 3) * (kTcRows * 128) +
-                                  (((chunk & 7) ^ (row & 7)) << 4);
-            st_shared_v4(addr, pack_bf16(p[0], p[1]), pack_bf16(p[2], p[3]), pack_bf16(p[4], p[5]),
-                         pack_bf16(p[6], p[7]));
+          } else {
+#pragma unroll
+            for (int chunk = 0; chunk < kTileTok / 8; ++chunk) {
+              float p[8];
+#pragma unroll
+              for (int x = 0; x < 8; ++x) {
+                const float e = ex2(fmaf(s[chunk * 8 + x], scale_log2, -m_safe));
+                p[x] = (chunk * 8 + x < vis) ? e : 0.0f;
+                ps[x] += p[x];
+              }
+              const uint32_t addr = p_row + (chunk >> 3) * (kTcRows * 128) +
+                                    (((chunk & 7) ^ (row & 7)) << 4);
+              st_shared_v4(addr, pack_bf16(p[0], p[1]), pack_bf16(p[2], p[3]), pack_bf16(p[4], p[5]),
+                           pack_bf16(p[6], p[7]));
+            }
           }
+          psum = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
         }
         l_run += psum;
         // last tile of the pair: V rows at or beyond the request's key count
@@ -706,6 +775,9 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         tc_fence_before();
         fence_async_smem();
         mbar_arrive(bar(B_P_FULL + b));
+#ifdef DSCALE_TRACE
+        busy_cycles += clock64() - tw1;
+#endif
       }
       if (!ok) break;
 #ifdef DSCALE_TRACE
@@ -794,6 +866,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     }
 #ifdef DSCALE_TRACE
     TRACE(60);
+    if (tid == 0) { trace[58] = wait_cycles; trace[59] = busy_cycles; trace[57] = it; }
 #endif
     // ---- end phase: publish what is left, merge the pairs this CTA is last to reach
     if (ok && (fin_i >= 0 || head_i >= 0)) {
