@@ -30,9 +30,10 @@
 //   warp 5     one thread issues tcgen05.mma: S = Q K^T (M64 N128 K128, bf16 in,
 //              fp32 in TMEM) for tile t, then O_t = P_{t-1} V_{t-1}; completion
 //              is signalled with tcgen05.commit on mbarriers.
-//   warps 0-3  softmax: thread (w, l < 16) owns row 16 w + l (TMEM lane 32 w + l),
-//              reads S with tcgen05.ld, keeps the running max / sum, writes P as
-//              bf16 into swizzled shared memory for the second MMA.  O stays in
+//   warps 0-3  softmax: warp w owns tile rows 16 w .. 16 w + 15 (TMEM lanes 32 w ..
+//              32 w + 15); tcgen05.ld.16x256b spreads them over all 32 lanes (a
+//              quad of threads per row).  They keep the running max / sum and
+//              write P as bf16 into swizzled shared memory for the second MMA.  O stays in
 //              TMEM for a whole run of tiles (the second MMA accumulates onto
 //              it); it is only rescaled in place when a row maximum outgrows its
 //              reference by 2^8, and read back once per run for the epilogue.
@@ -245,6 +246,29 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
 }
 __device__ __forceinline__ void tmem_st_wait() {
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+// 16 lanes x 128 columns per warp, spread over all 32 threads: thread t holds,
+// for each 8-column group n, v[4n], v[4n+1] = row t/4, columns 8n + 2(t%4) + {0,1}
+// and v[4n+2], v[4n+3] = row t/4 + 8, same columns (the m16n8 accumulator layout).
+__device__ __forceinline__ void tmem_ld_16x128(uint32_t taddr, float* v) {
+  uint32_t r[64];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int x = 0; x < 64; ++x) v[x] = __uint_as_float(r[x]);
+}
+__device__ __forceinline__ void tmem_st_16x128(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.16x256b.x16.b32 [%64], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63};"
+      ::"r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31])), "r"(__float_as_uint(v[32])), "r"(__float_as_uint(v[33])), "r"(__float_as_uint(v[34])), "r"(__float_as_uint(v[35])), "r"(__float_as_uint(v[36])), "r"(__float_as_uint(v[37])), "r"(__float_as_uint(v[38])), "r"(__float_as_uint(v[39])), "r"(__float_as_uint(v[40])), "r"(__float_as_uint(v[41])), "r"(__float_as_uint(v[42])), "r"(__float_as_uint(v[43])), "r"(__float_as_uint(v[44])), "r"(__float_as_uint(v[45])), "r"(__float_as_uint(v[46])), "r"(__float_as_uint(v[47])), "r"(__float_as_uint(v[48])), "r"(__float_as_uint(v[49])), "r"(__float_as_uint(v[50])), "r"(__float_as_uint(v[51])), "r"(__float_as_uint(v[52])), "r"(__float_as_uint(v[53])), "r"(__float_as_uint(v[54])), "r"(__float_as_uint(v[55])), "r"(__float_as_uint(v[56])), "r"(__float_as_uint(v[57])), "r"(__float_as_uint(v[58])), "r"(__float_as_uint(v[59])), "r"(__float_as_uint(v[60])), "r"(__float_as_uint(v[61])), "r"(__float_as_uint(v[62])), "r"(__float_as_uint(v[63])), "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void st_shared_b32(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -617,8 +641,12 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
            x += (long long)gridDim.x * kSoftmaxThreads)
         dst[x] = make_uint4(0, 0, 0, 0);
     }
-    const int row = warp * 16 + lane;                 // tile row m = 4 j + h_local
-    const int j_row = row >> 2, h_loc = row & 3;
+    // Thread t of warp w works on two tile rows, rA = 16 w + t / 4 and rB = rA + 8
+    // (tile row m = 4 j + h_local), and on the column pairs 8 n + 2 (t % 4) + {0, 1},
+    // n = 0..15: the layout tcgen05.ld.16x256b gives, so all 32 lanes carry 64 of
+    // the warp's 16 x 128 scores.  A row is shared by the 4 threads of a quad.
+    const int quad = lane & 3;
+    const int rowv[2] = {warp * 16 + (lane >> 2), warp * 16 + (lane >> 2) + 8};
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
     const uint32_t o_addr = t_lane + 256;
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
@@ -643,16 +671,53 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     auto wait_pv = [&](unsigned pt) -> bool {        // P.V of tile pt has completed
       return mbar_wait(bar(B_O_FULL + (pt & 1)), (pt >> 1) & 1, s_abort);
     };
+    auto quad_max = [](float v) {
+      v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+      return fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+    };
+    auto quad_sum = [](float v) {
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      return v + __shfl_xor_sync(0xffffffffu, v, 2);
+    };
+    // fold a partial (O row in shared memory at o_row, its (max, sum) = ml) into this
+    // thread's share of row h of acc
+    auto fold_row = [&](float* acc, int h, float& m_run, float& l_run, uint32_t o_row, float2 ml) {
+      const float m_tot = fmaxf(m_run, ml.x);
+      const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
+      const float w_me = ex2(m_run - m_s), w_o = ex2(ml.x - m_s);
+#pragma unroll
+      for (int n = 0; n < 16; ++n) {
+        const float2 v = ld_shared_v2f(o_row + (8 * n + 2 * quad) * 4);
+        acc[4 * n + 2 * h] = acc[4 * n + 2 * h] * w_me + v.x * w_o;
+        acc[4 * n + 2 * h + 1] = acc[4 * n + 2 * h + 1] * w_me + v.y * w_o;
+      }
+      l_run = l_run * w_me + ml.y * w_o;
+      m_run = m_tot;
+    };
+    // normalise and write this thread's share of row h: 16 column pairs
+    auto write_row = [&](const float* acc, int h, float l, int oi, int g) {
+      const float inv = 1.0f / l;
+      __nv_bfloat16* dst = out + ((size_t)(oi + (rowv[h] >> 2)) * Hq + g * 4 + (rowv[h] & 3)) * kD + 2 * quad;
+#pragma unroll
+      for (int n = 0; n < 16; ++n)
+        *reinterpret_cast<uint32_t*>(dst + 8 * n) = pack_bf16(acc[4 * n + 2 * h] * inv, acc[4 * n + 2 * h + 1] * inv);
+    };
 
     while (ok && sch.next(sg)) {
       const int ki = ws_ptr<int>(a.ws, L.k)[sg.i];
       const int oi = ws_ptr<int>(a.ws, L.offset)[sg.i];
       const int len = kv_len[sg.i];
-      const bool live = lane < 16 && j_row < ki;
-      const int pos = live ? ws_ptr<int>(a.ws, L.positions)[oi + j_row] : -1;
+      bool live[2];
+      int pos[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        live[h] = (rowv[h] >> 2) < ki;
+        pos[h] = live[h] ? ws_ptr<int>(a.ws, L.positions)[oi + (rowv[h] >> 2)] : -1;
+      }
       // O accumulates in TMEM relative to a reference maximum m_ref that is only
-      // raised (and O rescaled) when the row maximum outgrows it by 2^8
-      float m_ref = -INFINITY, l_run = 0.0f;
+      // raised (and O rescaled) when the row maximum outgrows it by 2^8.  l_part
+      // is this thread's share of the row sum (summed over the quad at the end).
+      float m_ref[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.0f, 0.0f};
 
       for (int t = sg.t0; t < sg.t1 && ok; ++t, ++it) {
         const int b = it & 1;
@@ -667,95 +732,87 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         const long long tw1 = clock64();
         wait_cycles += tw1 - tw0;
 #endif
-        float s[kTileTok];
-        tmem_ld128(t_lane + b * 128, s);
-        const int vis = min(kTileTok, max(0, pos + 1 - t * kTileTok));   // visible columns of this row
-        float mx = -INFINITY;
-        if (live) {
-          // eight independent running maxima: a single chain of 128 dependent
-          // fmax would cost its latency 128 times with one warp per scheduler
-          float m8[8];
+        float s[64];
+        tmem_ld_16x128(t_lane + b * 128, s);
+        int vis[2];
+        float mx[2];
+        bool need = false;
+        float factor[2] = {1.0f, 1.0f};
 #pragma unroll
-          for (int x = 0; x < 8; ++x) m8[x] = -INFINITY;
-          if (vis >= kTileTok) {
+        for (int h = 0; h < 2; ++h) {
+          vis[h] = min(kTileTok, max(0, pos[h] + 1 - t * kTileTok));     // visible columns of the row
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          if (vis[h] >= kTileTok) {
 #pragma unroll
-            for (int x = 0; x < kTileTok; ++x) m8[x & 7] = fmaxf(m8[x & 7], s[x]);
+            for (int n = 0; n < 16; ++n) {
+              m4[(2 * n) & 3] = fmaxf(m4[(2 * n) & 3], s[4 * n + 2 * h]);
+              m4[(2 * n + 1) & 3] = fmaxf(m4[(2 * n + 1) & 3], s[4 * n + 2 * h + 1]);
+            }
           } else {
 #pragma unroll
-            for (int x = 0; x < kTileTok; ++x) m8[x & 7] = (x < vis) ? fmaxf(m8[x & 7], s[x]) : m8[x & 7];
+            for (int n = 0; n < 16; ++n) {
+              const int col = 8 * n + 2 * quad;
+              if (col < vis[h]) m4[(2 * n) & 3] = fmaxf(m4[(2 * n) & 3], s[4 * n + 2 * h]);
+              if (col + 1 < vis[h]) m4[(2 * n + 1) & 3] = fmaxf(m4[(2 * n + 1) & 3], s[4 * n + 2 * h + 1]);
+            }
           }
-          mx = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])),
-                     fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
-        }
-        mx *= scale_log2;
-        float factor = 1.0f;
-        bool need = false;
-        if (t == sg.t0) {
-          m_ref = mx;                                   // the run's first P.V starts a fresh O
-        } else if (mx > m_ref + 8.0f) {
-          factor = ex2(m_ref - mx);
-          m_ref = mx;
-          l_run *= factor;
-          need = true;
+          mx[h] = quad_max(fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]))) * scale_log2;
+          if (t == sg.t0) {
+            m_ref[h] = mx[h];                          // the run's first P.V starts a fresh O
+          } else if (live[h] && mx[h] > m_ref[h] + 8.0f) {
+            factor[h] = ex2(m_ref[h] - mx[h]);
+            m_ref[h] = mx[h];
+            l_part[h] *= factor[h];
+            need = true;
+          }
         }
         if (__any_sync(0xffffffffu, need)) {
           // rescale this warp's O rows in TMEM before the next P.V accumulates
           ok = wait_pv(it - 1);
           if (!ok) break;
           tc_fence_after();
+          float o[64];
+          tmem_ld_16x128(o_addr, o);
 #pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            float o[32];
-            tmem_ld32(o_addr + ch * 32, o);
-#pragma unroll
-            for (int x = 0; x < 32; ++x) o[x] *= factor;
-            tmem_st32(o_addr + ch * 32, o);
+          for (int n = 0; n < 16; ++n) {
+            o[4 * n] *= factor[0]; o[4 * n + 1] *= factor[0];
+            o[4 * n + 2] *= factor[1]; o[4 * n + 3] *= factor[1];
           }
+          tmem_st_16x128(o_addr, o);
           tmem_st_wait();
         }
-        const float m_safe = (m_ref == -INFINITY) ? 0.0f : m_ref;
         // P[b] was last read by the P.V of tile it - 2
         if (it >= 2) { ok = wait_pv(it - 2); if (!ok) break; }
-        const uint32_t p_row = base + kOffP + b * kPBytes + row * 128;
-        float psum = 0.0f;
-        if (live) {
-          float ps[8];
+        const uint32_t p_base = base + kOffP + b * kPBytes + quad * 4;
 #pragma unroll
-          for (int x = 0; x < 8; ++x) ps[x] = 0.0f;
-          if (vis >= kTileTok) {
+        for (int h = 0; h < 2; ++h) {
+          const float m_safe = (m_ref[h] == -INFINITY) ? 0.0f : m_ref[h];
+          const uint32_t p_row = p_base + rowv[h] * 128;
+          const int sw = rowv[h] & 7;
+          float ps0 = 0.0f, ps1 = 0.0f;
+          if (vis[h] >= kTileTok) {
             // every column visible (all tiles but a pair's last one or two)
 #pragma unroll
-            for (int chunk = 0; chunk < kTileTok / 8; ++chunk) {      // 8 tokens = one 16-byte chunk
-              float p[8];
-#pragma unroll
-              for (int x = 0; x < 8; ++x) {
-                p[x] = ex2(fmaf(s[chunk * 8 + x], scale_log2, -m_safe));
-                ps[x] += p[x];
-              }
-              const uint32_t addr = p_row + (chunk >> 3) * (kTcRows * 128) +
-                                    (((chunk & 7) ^ (row & 7)) << 4);
-              st_shared_v4(addr, pack_bf16(p[0], p[1]), pack_bf16(p[2], p[3]), pack_bf16(p[4], p[5]),
-                           pack_bf16(p[6], p[7]));
+            for (int n = 0; n < 16; ++n) {
+              const float p0 = ex2(fmaf(s[4 * n + 2 * h], scale_log2, -m_safe));
+              const float p1 = ex2(fmaf(s[4 * n + 2 * h + 1], scale_log2, -m_safe));
+              ps0 += p0; ps1 += p1;
+              st_shared_b32(p_row + (n >> 3) * (kTcRows * 128) + (((n & 7) ^ sw) << 4), pack_bf16(p0, p1));
             }
-          } else {
+          } else if (live[h]) {
 #pragma unroll
-            for (int chunk = 0; chunk < kTileTok / 8; ++chunk) {
-              float p[8];
-#pragma unroll
-              for (int x = 0; x < 8; ++x) {
-                const float e = ex2(fmaf(s[chunk * 8 + x], scale_log2, -m_safe));
-                p[x] = (chunk * 8 + x < vis) ? e : 0.0f;
-                ps[x] += p[x];
-              }
-              const uint32_t addr = p_row + (chunk >> 3) * (kTcRows * 128) +
-                                    (((chunk & 7) ^ (row & 7)) << 4);
-              st_shared_v4(addr, pack_bf16(p[0], p[1]), pack_bf16(p[2], p[3]), pack_bf16(p[4], p[5]),
-                           pack_bf16(p[6], p[7]));
+            for (int n = 0; n < 16; ++n) {
+              const int col = 8 * n + 2 * quad;
+              float p0 = ex2(fmaf(s[4 * n + 2 * h], scale_log2, -m_safe));
+              float p1 = ex2(fmaf(s[4 * n + 2 * h + 1], scale_log2, -m_safe));
+              p0 = (col < vis[h]) ? p0 : 0.0f;
+              p1 = (col + 1 < vis[h]) ? p1 : 0.0f;
+              ps0 += p0; ps1 += p1;
+              st_shared_b32(p_row + (n >> 3) * (kTcRows * 128) + (((n & 7) ^ sw) << 4), pack_bf16(p0, p1));
             }
           }
-          psum = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
+          l_part[h] += ps0 + ps1;
         }
-        l_run += psum;
         // last tile of the pair: V rows at or beyond the request's key count
         // must be finite (0 x NaN would poison the row): zero them once the
         // copy has landed
@@ -789,9 +846,10 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       TRACE(tr); ++tr;
 #endif
       tc_fence_after();
-      float acc[kD];
-      tmem_ld128(o_addr, acc);
+      float acc[64];
+      tmem_ld_16x128(o_addr, acc);
       tc_fence_before();
+      float l_run[2] = {quad_sum(l_part[0]), quad_sum(l_part[1])};
 
       const int kind = run_kind(sg, sch.more());
       bool write_rows = (kind == RUN_WHOLE);
@@ -802,25 +860,15 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         const int fast = *s_fast;
         if (fast > 0) {
           // all other contributors' partials sit in ring slots 2 it, 2 it + 1, ...:
-          // fold them into this thread's row and finish the pair here
-          if (live) {
-            const uint32_t ml_base = base + kOffQ + ((seg + 1) & 1) * kQBytes;
-            for (int x = 0; x < fast; ++x) {
-              const uint32_t o_row = base + kOffKV + ((2 * it + x) % kStages) * kSlotBytes + row * (kD * 4);
-              const float2 ml = ld_shared_v2f(ml_base + (x * kTcRows + row) * 8);
-              const float m_tot = fmaxf(m_ref, ml.x);
-              const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
-              const float w_me = ex2(m_ref - m_s), w_o = ex2(ml.x - m_s);
+          // fold them into this thread's rows and finish the pair here
+          const uint32_t ml_base = base + kOffQ + ((seg + 1) & 1) * kQBytes;
+          for (int x = 0; x < fast; ++x) {
+            const uint32_t o_slot = base + kOffKV + ((2 * it + x) % kStages) * kSlotBytes;
 #pragma unroll
-              for (int d = 0; d < kD; d += 4) {
-                const float4 v = ld_shared_v4f(o_row + d * 4);
-                acc[d] = acc[d] * w_me + v.x * w_o;
-                acc[d + 1] = acc[d + 1] * w_me + v.y * w_o;
-                acc[d + 2] = acc[d + 2] * w_me + v.z * w_o;
-                acc[d + 3] = acc[d + 3] * w_me + v.w * w_o;
-              }
-              l_run = l_run * w_me + ml.y * w_o;
-              m_ref = m_tot;
+            for (int h = 0; h < 2; ++h) {
+              if (live[h])
+                fold_row(acc, h, m_ref[h], l_run[h], o_slot + rowv[h] * (kD * 4),
+                         ld_shared_v2f(ml_base + (x * kTcRows + rowv[h]) * 8));
             }
           }
           if (tid == 0) pair_cnt[sg.i * n_kv + sg.g] = 0;      // ready for the next launch
@@ -829,28 +877,27 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           store_partial = true;                                // ordinary path after the loop
         }
       }
-      if (write_rows && live) {
-        const float inv = 1.0f / l_run;
-        uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(oi + j_row) * Hq + sg.g * 4 + h_loc) * kD);
+      if (write_rows) {
 #pragma unroll
-        for (int d = 0; d < kD; d += 8) {
-          dst[d >> 3] = make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv),
-                                   pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
-                                   pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv),
-                                   pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
-        }
+        for (int h = 0; h < 2; ++h)
+          if (live[h]) write_row(acc, h, l_run[h], oi, sg.g);
       }
       if (store_partial) {
         // A run that covers only part of its pair: store the un-normalised partial.
         // Nothing in the main loop waits on global memory (a round trip costs
         // microseconds while every SM is streaming).
         const int slot_id = c * 2 + (sg.first_of_cta ? 0 : 1);
-        if (live) {
-          float4* po = reinterpret_cast<float4*>(part_o + ((size_t)slot_id * kTcRows + row) * kD);
 #pragma unroll
-          for (int d = 0; d < kD; d += 4) po[d >> 2] = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
-          *reinterpret_cast<float2*>(&part_ml[((size_t)slot_id * kTcRows + row) * 2]) =
-              make_float2(m_ref, l_run);
+        for (int h = 0; h < 2; ++h) {
+          if (live[h]) {
+            float* po = part_o + ((size_t)slot_id * kTcRows + rowv[h]) * kD + 2 * quad;
+#pragma unroll
+            for (int n = 0; n < 16; ++n)
+              *reinterpret_cast<float2*>(po + 8 * n) = make_float2(acc[4 * n + 2 * h], acc[4 * n + 2 * h + 1]);
+            if (quad == 0)
+              *reinterpret_cast<float2*>(&part_ml[((size_t)slot_id * kTcRows + rowv[h]) * 2]) =
+                  make_float2(m_ref[h], l_run[h]);
+          }
         }
         if (kind == RUN_PUBLISH) {
           mbar_arrive(bar(B_PART));                            // the publisher warp takes over
@@ -897,19 +944,19 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         if (ok && *s_head_last) { merge_i[n_merge] = head_i; merge_g[n_merge] = head_g; merge_n[n_merge] = head_n; ++n_merge; }
       }
       // Merge: all contributors' partials are bulk-copied into the (now idle) K/V
-      // ring, up to kStages at a time, and each thread combines its own row.
+      // ring, up to kStages at a time, and every thread folds its share of its rows.
       for (int x = 0; ok && x < n_merge; ++x) {
         __threadfence();
         const int pi = merge_i[x], pg = merge_g[x];
         const int ki = ws_ptr<int>(a.ws, L.k)[pi];
         const int oi = ws_ptr<int>(a.ws, L.offset)[pi];
-        const bool live = lane < 16 && j_row < ki;
+        const bool live[2] = {(rowv[0] >> 2) < ki, (rowv[1] >> 2) < ki};
         const long long p0 = ((long long)s_tile[pi] * n_kv) + (long long)pg * merge_n[x];
         const int c_lo = cta_of(p0, T, C), c_hi = cta_of(p0 + merge_n[x] - 1, T, C);
-        float acc[kD];
-        float m_run = -INFINITY, l_run = 0.0f;
+        float acc[64];
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
 #pragma unroll
-        for (int d = 0; d < kD; ++d) acc[d] = 0.0f;
+        for (int d = 0; d < 64; ++d) acc[d] = 0.0f;
         for (int cb = c_lo; cb <= c_hi && ok; cb += kStages) {
           const int nb = min(kStages, c_hi - cb + 1);
           ok = group_sync();                            // everybody is done with the ring slots
@@ -924,49 +971,34 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
                         kTcRows * kD * 4, bar(B_MERGE));
             }
           }
-          float2 ml[kStages];
+          float2 ml[kStages][2];
 #pragma unroll
           for (int y = 0; y < kStages; ++y) {
             const int cc = min(cb + y, c_hi);
             const int sid = cc * 2 + (slice_begin(cc, T, C) >= p0 ? 0 : 1);
-            ml[y] = live ? __ldcg(reinterpret_cast<const float2*>(&part_ml[((size_t)sid * kTcRows + row) * 2]))
-                         : make_float2(-INFINITY, 0.0f);
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+              ml[y][h] = live[h] ? __ldcg(reinterpret_cast<const float2*>(&part_ml[((size_t)sid * kTcRows + rowv[h]) * 2]))
+                                 : make_float2(-INFINITY, 0.0f);
           }
           ok = mbar_wait(bar(B_MERGE), merge_phase & 1, s_abort);
           ++merge_phase;
           if (!ok) break;
-          if (live) {
 #pragma unroll
-            for (int y = 0; y < kStages; ++y) {
-              if (y < nb) {
-                const uint32_t o_row = base + kOffKV + y * kSlotBytes + row * (kD * 4);
-                const float m_tot = fmaxf(m_run, ml[y].x);
-                const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
-                const float w_me = ex2(m_run - m_s), w_o = ex2(ml[y].x - m_s);
+          for (int y = 0; y < kStages; ++y) {
+            if (y < nb) {
 #pragma unroll
-                for (int d = 0; d < kD; d += 4) {
-                  const float4 v = ld_shared_v4f(o_row + d * 4);
-                  acc[d] = acc[d] * w_me + v.x * w_o;
-                  acc[d + 1] = acc[d + 1] * w_me + v.y * w_o;
-                  acc[d + 2] = acc[d + 2] * w_me + v.z * w_o;
-                  acc[d + 3] = acc[d + 3] * w_me + v.w * w_o;
-                }
-                l_run = l_run * w_me + ml[y].y * w_o;
-                m_run = m_tot;
-              }
+              for (int h = 0; h < 2; ++h)
+                if (live[h])
+                  fold_row(acc, h, m_run[h], l_run[h],
+                           base + kOffKV + y * kSlotBytes + rowv[h] * (kD * 4), ml[y][h]);
             }
           }
         }
-        if (ok && live) {
-          const float inv = 1.0f / l_run;
-          uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(oi + j_row) * Hq + pg * 4 + h_loc) * kD);
+        if (ok) {
 #pragma unroll
-          for (int d = 0; d < kD; d += 8) {
-            dst[d >> 3] = make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv),
-                                     pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
-                                     pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv),
-                                     pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
-          }
+          for (int h = 0; h < 2; ++h)
+            if (live[h]) write_row(acc, h, l_run[h], oi, pg);
         }
       }
     }
