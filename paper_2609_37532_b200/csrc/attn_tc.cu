@@ -393,7 +393,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     *s_dummy = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int x = tid; x <= n_bs; x += kThreads) s_tile[x] = ws_ptr<int>(a.ws, L.tile_prefix)[x];
   if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
                  ::"r"(smem_u32(s_tmem)) : "memory");
@@ -404,6 +403,13 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
   }
+  // Programmatic dependent launch: everything above (barriers, TMEM, descriptor
+  // prefetch) may overlap the tail of the preceding kernel in the stream; nothing
+  // that a preceding kernel may have written is read before this point.  The
+  // next kernel in the stream is allowed to start its own preamble right away.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  for (int x = tid; x <= n_bs; x += kThreads) s_tile[x] = ws_ptr<int>(a.ws, L.tile_prefix)[x];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -662,7 +668,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 #ifdef DSCALE_TRACE
     unsigned long long* trace = ws_ptr<unsigned long long>(a.ws, L.trace) + (size_t)c * 64;
     int tr = 2;
-    long long wait_cycles = 0, busy_cycles = 0;
+    long long wait_cycles = 0, busy_cycles = 0, c_ld = 0, c_max = 0, c_pvw = 0, c_exp = 0, c_fence = 0;
     if (tid == 0) { for (int x = 0; x < 64; ++x) trace[x] = 0; trace[0] = t_entry; trace[1] = gtime(); }
 #endif
     int head_i = -1, head_g = 0, head_n = 0;   // first run, published in the background
@@ -734,6 +740,10 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 #endif
         float s[64];
         tmem_ld_16x128(t_lane + b * 128, s);
+#ifdef DSCALE_TRACE
+        const long long tw2 = clock64();
+        c_ld += tw2 - tw1;
+#endif
         int vis[2];
         float mx[2];
         bool need = false;
@@ -781,8 +791,16 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           tmem_st_16x128(o_addr, o);
           tmem_st_wait();
         }
+#ifdef DSCALE_TRACE
+        const long long tw3 = clock64();
+        c_max += tw3 - tw2;
+#endif
         // P[b] was last read by the P.V of tile it - 2
         if (it >= 2) { ok = wait_pv(it - 2); if (!ok) break; }
+#ifdef DSCALE_TRACE
+        const long long tw4 = clock64();
+        c_pvw += tw4 - tw3;
+#endif
         const uint32_t p_base = base + kOffP + b * kPBytes + quad * 4;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -829,11 +847,16 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
             st_shared_v4(v_base + (hc >> 3) * kHalfSlot + r * 128 + ((hc & 7) << 4), 0, 0, 0, 0);
           }
         }
+#ifdef DSCALE_TRACE
+        const long long tw5 = clock64();
+        c_exp += tw5 - tw4;
+#endif
         tc_fence_before();
         fence_async_smem();
         mbar_arrive(bar(B_P_FULL + b));
 #ifdef DSCALE_TRACE
         busy_cycles += clock64() - tw1;
+        c_fence += clock64() - tw5;
 #endif
       }
       if (!ok) break;
@@ -913,7 +936,8 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     }
 #ifdef DSCALE_TRACE
     TRACE(60);
-    if (tid == 0) { trace[58] = wait_cycles; trace[59] = busy_cycles; trace[57] = it; }
+    if (tid == 0) { trace[58] = wait_cycles; trace[59] = busy_cycles; trace[57] = it;
+                    trace[52] = c_ld; trace[53] = c_max; trace[54] = c_pvw; trace[55] = c_exp; trace[56] = c_fence; }
 #endif
     // ---- end phase: publish what is left, merge the pairs this CTA is last to reach
     if (ok && (fin_i >= 0 || head_i >= 0)) {
@@ -1103,8 +1127,17 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t stream) {
       !kv_map(a.k_cache, a.n_kv_heads, a.num_pages, &tk) ||
       !kv_map(a.v_cache, a.n_kv_heads, a.num_pages, &tv))
     return cudaErrorNotSupported;
-  attn_tc_kernel<<<a.num_ctas, kThreads, kSmemBytes, stream>>>(a, L, tq, tk, tv);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.num_ctas);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, attn_tc_kernel, a, L, tq, tk, tv);
 }
 
 }  // namespace dscale
