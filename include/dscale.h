@@ -58,7 +58,8 @@ enum {
   DSCALE_ERR_INVALID_ARG = -1,   /* null / misaligned pointer, size out of range  */
   DSCALE_ERR_UNSUPPORTED = -2,   /* shape this build has no kernel for            */
   DSCALE_ERR_CUDA = -3,          /* a CUDA runtime / driver call failed           */
-  DSCALE_ERR_WORKSPACE = -4      /* workspace too small or not initialised        */
+  DSCALE_ERR_WORKSPACE = -4,     /* workspace too small or not initialised        */
+  DSCALE_ERR_TOO_LARGE = -5      /* size beyond a fixed built-in capacity         */
 };
 
 /* bits of the device status word (0 = OK; bits are OR-ed, sticky until
@@ -212,6 +213,35 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
                             int n_q_heads, int n_kv_heads, float sm_scale, const float* logits,
                             int64_t ld, int vocab, int32_t* h_accept_len, int32_t* h_next_anchor,
                             int32_t* h_out_tokens, int32_t* h_out_len, void* stream);
+
+/*
+ * Greedy prefix verification for callers that can neither allocate nor keep a
+ * workspace.  (The paper has no counterpart to this call: it exists for
+ * deployment reasons only.)  Typical users: a serving loop in which a cudaMalloc
+ * would stall every stream of the device, or a plug-in that only receives input
+ * and output pointers from its host runtime.  Same result as dscale_accept, but
+ * the lengths, offsets and packed tokens are passed in explicitly and the
+ * scratch of the row argmax lives in a fixed __device__ array inside the
+ * library (about 66 KB per GPU, held until the process exits).  The call
+ * allocates nothing and frees nothing.
+ *
+ *   n_live [1], k [n_bs], offset [n_bs + 1], tokens [8 n_bs]   int32, device:
+ *         as produced by dscale_alloc_verify (workspace fields N_LIVE, K,
+ *         OFFSET, TOKENS) or by the caller
+ *   logits, ld, vocab and the four outputs: as in dscale_accept
+ *
+ * Limits and rules: n_bs <= DSCALE_ACCEPT_STATIC_MAX_NBS, otherwise
+ * DSCALE_ERR_TOO_LARGE is returned and nothing is enqueued.  All calls on a GPU
+ * share the one scratch array, so two calls that may run at the same time on
+ * that GPU (different streams or threads) race: serialise them.  The first call
+ * on each device looks up the array's address; make that call before any stream
+ * capture begins.
+ */
+#define DSCALE_ACCEPT_STATIC_MAX_NBS 64
+int dscale_accept_static(int n_bs, const int32_t* n_live, const int32_t* k, const int32_t* offset,
+                         const int32_t* tokens, const float* logits, int64_t ld, int vocab,
+                         int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
+                         int32_t* out_len, void* stream);
 
 /*
  * Device address of a workspace field (see DSCALE_WS_*), for tests and for

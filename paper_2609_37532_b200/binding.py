@@ -42,6 +42,8 @@ lib.dscale_verify_step_host.restype = _i
 lib.dscale_verify_step_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _i, _vp,
                                         C.POINTER(LayerPtrs), _i, _i, _i, _f, _vp, _i64, _i,
                                         _vp, _vp, _vp, _vp, _vp]
+lib.dscale_accept_static.restype = _i
+lib.dscale_accept_static.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _i64, _i, _vp, _vp, _vp, _vp, _vp]
 lib.dscale_ws_field.restype = _vp
 lib.dscale_ws_field.argtypes = [_vp, _i, _i]
 lib.dscale_launches_per_call.restype = _i
@@ -49,7 +51,8 @@ lib.dscale_launches_per_call.argtypes = [_i]
 
 WS_FIELDS = dict(status=0, k=1, offset=2, q_start=3, q_end=4, tokens=5, positions=6, kv_refs=7,
                  row_req=8, top1=9, k0=10, n_live=11)
-_ERR = {-1: "invalid argument", -2: "unsupported shape", -3: "CUDA error", -4: "workspace"}
+_ERR = {-1: "invalid argument", -2: "unsupported shape", -3: "CUDA error", -4: "workspace",
+        -5: "size beyond the built-in capacity"}
 
 
 class DScaleError(RuntimeError):
@@ -199,3 +202,20 @@ class HostStep:
             ws.n_q_heads, ws.n_kv_heads, self.sm_scale, _ptr(self.logits),
             self.logits.stride(0), self.vocab, _ptr(self.h_accept_len), _ptr(self.h_next_anchor),
             _ptr(self.h_out_tokens), _ptr(self.h_out_len), _stream()), "dscale_verify_step_host")
+
+
+def accept_static(n_bs: int, n_live, k, offset, tokens, logits, vocab: int, accept_len,
+                  next_anchor, out_tokens, out_len):
+    """dscale_accept_static: acceptance without a workspace and without any
+    allocation (the scratch is a fixed array inside the library).  For callers
+    that cannot call cudaMalloc on their hot path.  Calls on one GPU must not
+    overlap; make the first call on a device outside stream capture."""
+    _need(logits, torch.float32, "logits")
+    for n, t in (("n_live", n_live), ("k", k), ("offset", offset), ("tokens", tokens),
+                 ("accept_len", accept_len), ("next_anchor", next_anchor),
+                 ("out_tokens", out_tokens), ("out_len", out_len)):
+        _need(t, torch.int32, n)
+    _check(lib.dscale_accept_static(n_bs, _ptr(n_live), _ptr(k), _ptr(offset), _ptr(tokens),
+                                    _ptr(logits), logits.stride(0), vocab, _ptr(accept_len),
+                                    _ptr(next_anchor), _ptr(out_tokens), _ptr(out_len), _stream()),
+           "dscale_accept_static")
