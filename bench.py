@@ -121,33 +121,37 @@ def algorithmic_bytes(cfg, req, k):
 
 
 # ------------------------------------------------------------------ CPU oracle
-def oracle_step_sample(cfg, req, kc0, vc0, q0_unpacked, logits_unpacked):
+def oracle_step_sample(cfg, req, kvs, q_unpacked, logits_unpacked):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload:
-    allocation and acceptance in full, attention on ONE layer (all requests),
-    and extrapolates the step time to cfg.layers layers.  Returns
-    (tokens_per_s, seconds of CPU work, description)."""
+    allocation and acceptance in full, attention on the first len(kvs) layers
+    (all requests), and scales the attention time to cfg.layers layers.
+    Returns (tokens_per_s, seconds of CPU work, description)."""
     from oracle import accept as OC
     from oracle import dvl_alloc as OA
     from oracle import verify_attn as OV
     t0 = time.perf_counter()
     alloc = OA.dvl_alloc(req["n_bs"], req["n_live"], req["scores"], req["draft_tokens"],
                          req["ctx_len"], req["block_table"])
-    t1 = time.perf_counter()
-    qp = rows_to_packed(q0_unpacked, alloc["k"], alloc["offset"], req["n_live"], 8 * req["n_bs"])
+    t_alloc = time.perf_counter() - t0
     lp = rows_to_packed(logits_unpacked, alloc["k"], alloc["offset"], req["n_live"], 8 * req["n_bs"])
-    qf, kf, vf, lf = qp.float().numpy(), kc0.float().numpy(), vc0.float().numpy(), lp.numpy()
-    t2 = time.perf_counter()
-    OV.verify_attn(qf, kf, vf, req["block_table"], req["ctx_len"], alloc["k"], alloc["offset"],
-                   req["n_live"], cfg.n_q_heads, cfg.n_kv_heads, SCALE)
+    lf = lp.numpy()
+    t_attn = 0.0
+    for (kc, vc), qu in zip(kvs, q_unpacked):
+        qp = rows_to_packed(qu, alloc["k"], alloc["offset"], req["n_live"], 8 * req["n_bs"])
+        qf, kf, vf = qp.float().numpy(), kc.float().numpy(), vc.float().numpy()
+        t2 = time.perf_counter()
+        OV.verify_attn(qf, kf, vf, req["block_table"], req["ctx_len"], alloc["k"], alloc["offset"],
+                       req["n_live"], cfg.n_q_heads, cfg.n_kv_heads, SCALE)
+        t_attn += time.perf_counter() - t2
     t3 = time.perf_counter()
     res = OC.accept(lf, cfg.vocab, alloc["tokens"], alloc["k"], alloc["offset"], req["n_live"],
                     req["n_bs"])
-    t4 = time.perf_counter()
+    t_acc = time.perf_counter() - t3
     tokens = int(res["out_len"].sum())
-    step = (t1 - t0) + cfg.layers * (t3 - t2) + (t4 - t3)
-    work = (t1 - t0) + (t3 - t2) + (t4 - t3)
-    desc = (f"allocation and acceptance in full, attention on layer 0 of {cfg.layers} "
-            f"(all {req['n_live']} requests), attention time x {cfg.layers}")
+    step = t_alloc + cfg.layers * (t_attn / len(kvs)) + t_acc
+    work = t_alloc + t_attn + t_acc
+    desc = (f"allocation and acceptance in full, attention on the first {len(kvs)} of {cfg.layers} "
+            f"layers (all {req['n_live']} requests), attention time scaled to {cfg.layers} layers")
     return tokens / step, work, desc
 
 
@@ -166,13 +170,14 @@ def run_reference(args, rank):
         return
     cfg = CONFIGS[args.workload]
     req = make_requests(cfg)
-    kc, vc = make_kv_layer(req, 0, poison=False)
-    qu = make_q_unpacked(req, 0)
+    n_l = min(cfg.layers, args.cpu_layers)
+    kvs = [make_kv_layer(req, l, poison=False) for l in range(n_l)]
+    qus = [make_q_unpacked(req, l) for l in range(n_l)]
     lu = make_logits_unpacked(req)
     vals, work = [], 0.0
     desc = ""
     for s in range(args.warmup + args.steps):
-        v, w, desc = oracle_step_sample(cfg, req, kc, vc, qu, lu)
+        v, w, desc = oracle_step_sample(cfg, req, kvs, qus, lu)
         if s >= args.warmup:
             vals.append(v); work += w
     value = float(np.mean(vals))
@@ -281,20 +286,29 @@ def run_ours(args, rank, world, local_rank):
         barrier()
         ms_total = e0.elapsed_time(e1)
 
-        # ---- timed region 2: same steps as direct launches, with events around the
-        # attention launches, for the per-kernel roofline ----
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
-               torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-        for s in range(args.steps):
-            do_alloc()
-            ev[s][0].record(stream)
+        # ---- timed region 2: the dominant kernel alone, for its roofline: the L
+        # attention launches of a step captured as their own graph (same launch
+        # configuration as in the step), K replays, CUDA events around each ----
+        g_attn = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_attn, stream=stream):
             do_attn()
-            ev[s][1].record(stream)
-            do_accept()
-            ev[s][2].record(stream)
+        g_attn.replay()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(args.steps)]
         barrier()
-        attn_ms = float(np.mean([a.elapsed_time(b) for a, b, _ in ev])) / max(1, cfg.layers)
-        accept_ms = float(np.mean([b.elapsed_time(c) for _, b, c in ev]))
+        for s in range(args.steps):
+            ev[s][0].record(stream)
+            g_attn.replay()
+            ev[s][1].record(stream)
+        barrier()
+        attn_ms = float(np.mean([a.elapsed_time(b) for a, b in ev])) / max(1, cfg.layers)
+        ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ea.record(stream)
+        for _ in range(args.steps):
+            do_accept()
+        eb.record(stream)
+        barrier()
+        accept_ms = ea.elapsed_time(eb) / args.steps
 
         # ---- timed region 3: end to end through the host-buffer C ABI call ----
         hs = P.HostStep(ws, req["max_pages"], req["num_pages"], layers, logits, cfg.vocab, SCALE)
@@ -363,10 +377,11 @@ def run_ours(args, rank, world, local_rank):
             "clocks": clocks,
         }
         if world == 1 and not args.no_cpu_baseline:
-            kc0, vc0 = layers[0][1].cpu(), layers[0][2].cpu()
-            qu0 = make_q_unpacked(req, 0, device=str(dev)).cpu()
+            n_l = min(cfg.layers, args.cpu_layers)
+            kvs = [(layers[l][1].cpu(), layers[l][2].cpu()) for l in range(n_l)]
+            qus = [make_q_unpacked(req, l, device=str(dev)).cpu() for l in range(n_l)]
             lu_cpu = make_logits_unpacked(req, device=str(dev)).cpu()
-            v, work, desc = oracle_step_sample(cfg, req, kc0, vc0, qu0, lu_cpu)
+            v, work, desc = oracle_step_sample(cfg, req, kvs, qus, lu_cpu)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                     "sample": desc, "cpu_seconds": work}
         print(json.dumps(line))
@@ -377,14 +392,19 @@ def run_ours(args, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen3_8b_step", choices=list(CONFIGS))
     ap.add_argument("--attn", default="tensor", choices=["tensor", "simt"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-layers", type=int, default=0,
+                    help="layers of attention the CPU oracle is timed on (its time is scaled to all "
+                         "layers); default 12 for the cpu_baseline leg, 2 per step for --impl reference")
     args = ap.parse_args()
+    if args.cpu_layers <= 0:
+        args.cpu_layers = 12 if args.impl == "ours" else 2
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
