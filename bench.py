@@ -198,6 +198,24 @@ def run_reference(args, rank):
 
 
 # ------------------------------------------------------------------- GPU bench
+def replica_config(base, rank: int):
+    """Every rank is an independent replica with its own seeded batch."""
+    return small_variant(base, seed=base.seed + 1000 * rank)
+
+
+def aggregate(dist, t):
+    """t = [ms_per_step, attn_ms, e2e_seconds, tokens_per_step, e2e_tokens] of this rank.
+    Times are the maximum over ranks, token counts the sum (whole-job throughput)."""
+    if dist is not None:
+        tmax = t.clone()
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        tsum = t.clone()
+        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+    else:
+        tmax = tsum = t
+    return float(tmax[0]), float(tmax[1]), float(tmax[2]), float(tsum[3]), float(tsum[4])
+
+
 def run_ours(args, rank, world, local_rank):
     import paper_2609_37532_b200 as P
     torch.cuda.set_device(local_rank)
@@ -209,7 +227,7 @@ def run_ours(args, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=dev)
 
     base = CONFIGS[args.workload]
-    cfg = small_variant(base, seed=base.seed + 1000 * rank)      # every replica has its own batch
+    cfg = replica_config(base, rank)
     if args.layers:
         cfg = small_variant(cfg, layers=args.layers)
     req = make_requests(cfg)
@@ -333,13 +351,7 @@ def run_ours(args, rank, world, local_rank):
     ms_step = ms_total / args.steps
     t = torch.tensor([ms_step, attn_ms, e2e_s, float(tokens_per_step), float(e2e_tokens)],
                      dtype=torch.float64, device=dev)
-    if dist is not None:
-        tmax = t.clone(); dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = t.clone(); dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-    else:
-        tmax = tsum = t
-    ms_step, attn_ms, e2e_s = float(tmax[0]), float(tmax[1]), float(tmax[2])
-    tokens_all, e2e_tokens_all = float(tsum[3]), float(tsum[4])
+    ms_step, attn_ms, e2e_s, tokens_all, e2e_tokens_all = aggregate(dist, t)
     value = tokens_all / (ms_step * 1e-3)
     e2e_value = e2e_tokens_all / e2e_s
 
