@@ -403,17 +403,22 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
   }
-  // Programmatic dependent launch: everything above (barriers, TMEM, descriptor
-  // prefetch) may overlap the tail of the preceding kernel in the stream; nothing
-  // that a preceding kernel may have written is read before this point.  The
-  // next kernel in the stream is allowed to start its own preamble right away.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Programmatic dependent launch.  This kernel may become resident while the
+  // preceding kernel of the stream is still finishing on other SMs.  Until
+  // griddepcontrol.wait it only touches data that the immediately preceding
+  // kernel cannot be writing: the allocation's metadata in the workspace (the
+  // allocation kernel never lets its dependents start early), the block table,
+  // and K/V pages that lie wholly below the committed context (the cache is
+  // append-only).  Q, the window's K/V pages and every write (outputs, split-KV
+  // scratch) come after the wait.  The next kernel may start its own preamble
+  // as soon as SMs free up.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   for (int x = tid; x <= n_bs; x += kThreads) s_tile[x] = ws_ptr<int>(a.ws, L.tile_prefix)[x];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  if (warp != 4) asm volatile("griddepcontrol.wait;" ::: "memory");   // the producer waits later
 
   const long long T = (long long)s_tile[n_bs] * n_kv;
   // with fewer tiles than CTAs only the first T CTAs get a (one-tile) slice, so
@@ -430,21 +435,13 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     unsigned u = 0;            // ring sequence number: K of tile it -> 2 it, V -> 2 it + 1
     int seg = 0;
     bool ok = true;
+    bool waited = false;       // griddepcontrol.wait done
+    // lane l copies page l / 2, column half l % 2 (lanes 0..15)
+    const int pg_l = lane >> 1, half = lane & 1;
     while (ok && sch.next(sg)) {
       const int qb = seg & 1;
-      ok = mbar_wait(bar(B_Q_EMPTY + qb), ((seg >> 1) & 1) ^ 1, s_abort);
-      if (!ok) break;
-      if (lane == 0) {
-        const int row0 = ws_ptr<int>(a.ws, L.offset)[sg.i];
-        mbar_expect_tx(bar(B_Q_FULL + qb), kQBytes);
-        tma_load_4d(base + kOffQ + qb * kQBytes, &tm_q, bar(B_Q_FULL + qb), 0, 0, sg.g * 4, row0);
-        tma_load_4d(base + kOffQ + qb * kQBytes + kQBytes / 2, &tm_q, bar(B_Q_FULL + qb), 0, 1,
-                    sg.g * 4, row0);
-      }
       const int len = kv_len[sg.i];
       const int* bt = a.block_table + (size_t)sg.i * a.max_pages;
-      // lane l copies page l / 2, column half l % 2 (lanes 0..15)
-      const int pg_l = lane >> 1, half = lane & 1;
       auto fetch_page = [&](int t) -> int {
         const int p = t * (kTileTok / kPage) + pg_l;
         int id = 0;
@@ -454,17 +451,13 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         }
         return id;
       };
-      int page_next = fetch_page(sg.t0);
-      for (int t = sg.t0; t < sg.t1 && ok; ++t) {
-        const int page = page_next;
-        if (t + 1 < sg.t1) page_next = fetch_page(t + 1);
+      auto issue_tile = [&](int t, int page) -> bool {       // K then V of key tile t into the ring
         const int valid_tok = min(kTileTok, len - t * kTileTok);
         const int n_pages = (valid_tok + kPage - 1) / kPage;
 #pragma unroll
         for (int which = 0; which < 2; ++which, ++u) {
           const int slot = u % kStages;
-          ok = mbar_wait(bar(B_KV_EMPTY + slot), ((u / kStages) & 1) ^ 1, s_abort);
-          if (!ok) break;
+          if (!mbar_wait(bar(B_KV_EMPTY + slot), ((u / kStages) & 1) ^ 1, s_abort)) return false;
           if (lane == 0) mbar_expect_tx(bar(B_KV_FULL + slot), n_pages * 2 * kPageBoxBytes);
           __syncwarp();
           if (lane < 16 && pg_l < n_pages) {
@@ -472,6 +465,38 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
                         which == 0 ? &tm_k : &tm_v, bar(B_KV_FULL + slot), 0, half, 0, sg.g, page);
           }
         }
+        return true;
+      };
+      int t_first = sg.t0;
+      if (!waited) {
+        // before the grid dependency is resolved: up to two key tiles that lie wholly
+        // below the committed context of the first run's request
+        const int ctx0 = len - ws_ptr<int>(a.ws, L.k)[sg.i];
+        while (ok && t_first < sg.t1 && t_first < sg.t0 + 2 && (t_first + 1) * kTileTok <= ctx0) {
+          ok = issue_tile(t_first, fetch_page(t_first));
+          ++t_first;
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        waited = true;
+#ifdef DSCALE_TRACE
+        if (lane == 0) ws_ptr<unsigned long long>(a.ws, L.trace)[(size_t)c * 64 + 63] = gtime();
+#endif
+        if (!ok) break;
+      }
+      ok = mbar_wait(bar(B_Q_EMPTY + qb), ((seg >> 1) & 1) ^ 1, s_abort);
+      if (!ok) break;
+      if (lane == 0) {
+        const int row0 = ws_ptr<int>(a.ws, L.offset)[sg.i];
+        mbar_expect_tx(bar(B_Q_FULL + qb), kQBytes);
+        tma_load_4d(base + kOffQ + qb * kQBytes, &tm_q, bar(B_Q_FULL + qb), 0, 0, sg.g * 4, row0);
+        tma_load_4d(base + kOffQ + qb * kQBytes + kQBytes / 2, &tm_q, bar(B_Q_FULL + qb), 0, 1,
+                    sg.g * 4, row0);
+      }
+      int page_next = t_first < sg.t1 ? fetch_page(t_first) : 0;
+      for (int t = t_first; t < sg.t1 && ok; ++t) {
+        const int page = page_next;
+        if (t + 1 < sg.t1) page_next = fetch_page(t + 1);
+        ok = issue_tile(t, page);
       }
 #ifndef DSCALE_STREAM_ONLY
       if (ok && run_kind(sg, sch.more()) == RUN_TAIL) {
@@ -513,6 +538,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 #endif
       ++seg;
     }
+    if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");
     // on an aborted run, let the copies already issued land before the CTA's
     // shared memory is released (bounded, like every other wait)
     if (!ok) {
@@ -1039,6 +1065,9 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
   }
+#ifdef DSCALE_TRACE
+  if (tid == 0) ws_ptr<unsigned long long>(a.ws, L.trace)[(size_t)c * 64 + 62] = gtime();
+#endif
 }
 
 // ------------------------------------------------------------ host: tensor maps
