@@ -388,6 +388,30 @@ def run_ours(args, rank, world, local_rank):
                                           P.lib.dscale_launches_per_call(2)),
             "clocks": clocks,
         }
+        if world == 1 and not args.no_padded:
+            # the in-repo comparison: unpacked W = 16, one 128-row tile per (request, q-head)
+            with torch.cuda.stream(stream):
+                qus = [make_q_unpacked(req, l, device=str(dev)) for l in range(cfg.layers)]
+                ous = [torch.empty_like(q) for q in qus]
+
+                def do_padded():
+                    for l, (q, kc, vc, o) in enumerate(layers):
+                        P.verify_attn_padded(ws, qus[l], kc, vc, d_bt, d_ctx, SCALE, ous[l])
+                do_padded()
+                pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                n_rep = max(1, min(args.steps, 5))
+                pa.record(stream)
+                for _ in range(n_rep):
+                    do_padded()
+                pb.record(stream)
+                torch.cuda.synchronize()
+                pad_us = 1e3 * pa.elapsed_time(pb) / n_rep / max(1, cfg.layers)
+            line["padded_baseline"] = {
+                "what": "unpacked W=16 verify attention, 128-row tile per (request, q-head), 16N rows",
+                "attn_us_per_launch": pad_us, "packed_attn_us_per_launch": attn_ms * 1e3,
+                "attn_speedup_packed_vs_padded": pad_us / (attn_ms * 1e3)}
+            del qus, ous
         if world == 1 and not args.no_cpu_baseline:
             n_l = min(cfg.layers, args.cpu_layers)
             kvs = [(layers[l][1].cpu(), layers[l][2].cpu()) for l in range(n_l)]
@@ -411,6 +435,7 @@ def main():
     ap.add_argument("--attn", default="tensor", choices=["tensor", "simt"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-padded", action="store_true", help="skip the padded comparison kernel")
     ap.add_argument("--cpu-layers", type=int, default=0,
                     help="layers of attention the CPU oracle is timed on (its time is scaled to all "
                          "layers); default 12 for the cpu_baseline leg, 2 per step for --impl reference")

@@ -163,6 +163,24 @@ int dscale_verify_attn_simt(void* ws, int n_bs, const void* q, const void* k_cac
                             void* out, void* stream);
 
 /*
+ * Comparison baseline, not part of the method: verify attention the way the
+ * paper describes the native path (Section 2.1) -- every live request verifies
+ * all W = 16 slots, and each (request, q-head) owns one 128-row tile of which
+ * 16 rows are live (Eq. 2: 112 masked rows, 87.5 %).  K/V are streamed once per
+ * q-head.  Same kernel machinery as dscale_verify_attn otherwise.
+ *
+ *   q_unpacked, out_unpacked   bf16 [n_bs][16][n_q_heads][128]; row j of request i
+ *                 sees the logical keys 0 .. ctx_len[i] + j; requests >= N are
+ *                 written as zero
+ *   ctx_len       int32 [n_bs], as given to dscale_alloc_verify (N is taken from
+ *                 the workspace, so an allocation must have run)
+ */
+int dscale_verify_attn_padded(void* ws, int n_bs, const void* q_unpacked, const void* k_cache,
+                              const void* v_cache, const int32_t* block_table, int max_pages,
+                              int num_pages, const int32_t* ctx_len, int n_q_heads,
+                              int n_kv_heads, float sm_scale, void* out_unpacked, void* stream);
+
+/*
  * Greedy prefix verification and output building ("Prefix verifier" paragraph;
  * Algorithm 2, lines 21-26).  top1[s] = first index of the maximum of
  * logits[s][0..vocab) for s < M_live (a NaN never counts as a maximum).
@@ -251,7 +269,7 @@ int dscale_accept_static(int n_bs, const int32_t* n_live, const int32_t* k, cons
 const int32_t* dscale_ws_field(const void* ws, int n_bs, int field);
 
 /* Number of kernels the three stage calls enqueue (for launch accounting):
- * which = 0 alloc, 1 attention, 2 accept, 3 attention (simt). */
+ * which = 0 alloc, 1 attention, 2 accept, 3 attention (simt), 4 attention (padded). */
 int dscale_launches_per_call(int which);
 
 #ifdef __cplusplus

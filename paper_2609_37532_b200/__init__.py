@@ -11,7 +11,7 @@ _build()          # no-op when libdscale.so is newer than its sources; raises if
 
 from .binding import (  # noqa: E402
     DScaleError, HostStep, VerifyWorkspace, accept, accept_static, alloc_verify, lib, verify_attn,
-                      verify_attn_simt, WS_FIELDS)
+                      verify_attn_padded, verify_attn_simt, WS_FIELDS)
 
 __all__ = ["DScaleError", "HostStep", "VerifyWorkspace", "accept", "accept_static", "alloc_verify", "lib", "verify_attn",
-           "verify_attn_simt", "WS_FIELDS"]
+           "verify_attn_padded", "verify_attn_simt", "WS_FIELDS"]

@@ -42,6 +42,8 @@ lib.dscale_verify_step_host.restype = _i
 lib.dscale_verify_step_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _i, _vp,
                                         C.POINTER(LayerPtrs), _i, _i, _i, _f, _vp, _i64, _i,
                                         _vp, _vp, _vp, _vp, _vp]
+lib.dscale_verify_attn_padded.restype = _i
+lib.dscale_verify_attn_padded.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i, _i, _vp, _i, _i, _f, _vp, _vp]
 lib.dscale_accept_static.restype = _i
 lib.dscale_accept_static.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _i64, _i, _vp, _vp, _vp, _vp, _vp]
 lib.dscale_ws_field.restype = _vp
@@ -219,3 +221,16 @@ def accept_static(n_bs: int, n_live, k, offset, tokens, logits, vocab: int, acce
                                     _ptr(logits), logits.stride(0), vocab, _ptr(accept_len),
                                     _ptr(next_anchor), _ptr(out_tokens), _ptr(out_len), _stream()),
            "dscale_accept_static")
+
+
+def verify_attn_padded(ws, q_unpacked, k_cache, v_cache, block_table, ctx_len, sm_scale, out_unpacked):
+    """The comparison baseline: unpacked W = 16, one 128-row tile per (request, q-head)."""
+    _need(q_unpacked, torch.bfloat16, "q_unpacked"); _need(out_unpacked, torch.bfloat16, "out_unpacked")
+    _need(k_cache, torch.bfloat16, "k_cache"); _need(v_cache, torch.bfloat16, "v_cache")
+    _need(block_table, torch.int32, "block_table"); _need(ctx_len, torch.int32, "ctx_len")
+    assert q_unpacked.shape == (ws.n_bs, 16, ws.n_q_heads, 128) and out_unpacked.shape == q_unpacked.shape
+    _check(lib.dscale_verify_attn_padded(C.c_void_p(ws.ptr), ws.n_bs, _ptr(q_unpacked), _ptr(k_cache),
+                                         _ptr(v_cache), _ptr(block_table), block_table.shape[1],
+                                         k_cache.shape[0], _ptr(ctx_len), ws.n_q_heads, ws.n_kv_heads,
+                                         float(sm_scale), _ptr(out_unpacked), _stream()),
+           "dscale_verify_attn_padded")

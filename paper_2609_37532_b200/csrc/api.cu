@@ -11,6 +11,7 @@
 namespace dscale {
 cudaError_t attn_simt_prepare();
 cudaError_t attn_tc_prepare();
+cudaError_t attn_padded_prepare();
 }
 
 namespace {
@@ -64,6 +65,7 @@ int dscale_workspace_init(void* ws, size_t bytes, int n_bs, int n_q_heads, int n
   if (cudaMemsetAsync(ws, 0, L.part_o, (cudaStream_t)stream) != cudaSuccess) return DSCALE_ERR_CUDA;
   if (attn_simt_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
   if (attn_tc_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
+  if (attn_padded_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
   std::lock_guard<std::mutex> lk(g_mu);
   g_ws[ws] = WsInfo{bytes, n_bs, n_q_heads, n_kv_heads, num_sms};
   return DSCALE_OK;
@@ -126,6 +128,22 @@ int dscale_verify_attn_simt(void* ws, int n_bs, const void* q, const void* k_cac
                        n_q_heads, n_kv_heads, sm_scale, out, &a);
   if (rc != DSCALE_OK) return rc;
   return launch_attn_simt(a, (cudaStream_t)stream) == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
+}
+
+int dscale_verify_attn_padded(void* ws, int n_bs, const void* q_unpacked, const void* k_cache,
+                              const void* v_cache, const int32_t* block_table, int max_pages,
+                              int num_pages, const int32_t* ctx_len, int n_q_heads,
+                              int n_kv_heads, float sm_scale, void* out_unpacked, void* stream) {
+  if (!ctx_len) return DSCALE_ERR_INVALID_ARG;
+  AttnArgs a;
+  int rc = attn_common(ws, n_bs, q_unpacked, k_cache, v_cache, block_table, max_pages, num_pages,
+                       n_q_heads, n_kv_heads, sm_scale, out_unpacked, &a);
+  if (rc != DSCALE_OK) return rc;
+  cudaError_t e = launch_attn_padded(ws, n_bs, q_unpacked, k_cache, v_cache, block_table, max_pages,
+                                     num_pages, ctx_len, n_q_heads, n_kv_heads, sm_scale,
+                                     out_unpacked, a.num_ctas, (cudaStream_t)stream);
+  if (e == cudaErrorNotSupported) return DSCALE_ERR_UNSUPPORTED;
+  return e == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
 }
 
 int dscale_accept(void* ws, int n_bs, const float* logits, int64_t ld, int vocab,
@@ -249,6 +267,7 @@ int dscale_launches_per_call(int which) {
     case 1: return 1;   // attn_tc_kernel (cut pairs are merged inside it)
     case 2: return 1;   // accept_kernel
     case 3: return 1;   // attn_simt_kernel
+    case 4: return 1;   // attn_padded_kernel
     default: return 0;
   }
 }

@@ -58,4 +58,11 @@ cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t stream);
 // returns cudaErrorNotSupported if the driver entry point for tensor maps is missing
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t stream);
 
+// comparison baseline: unpacked W = 16, one 128-row tile per (request, q-head)
+cudaError_t launch_attn_padded(void* ws, int n_bs, const void* q_unpacked, const void* k_cache,
+                               const void* v_cache, const int32_t* block_table, int max_pages,
+                               int num_pages, const int32_t* ctx_len, int n_q_heads,
+                               int n_kv_heads, float sm_scale, void* out_unpacked, int num_ctas,
+                               cudaStream_t stream);
+
 }  // namespace dscale

@@ -28,7 +28,7 @@ enum HdrWord {
 
 struct WsLayout {
   size_t hdr, k, k0, offset, q_start, q_end, tokens, positions, kv_refs, row_req, top1,
-      kv_len, tile_prefix, qscores, amax_val, amax_idx, pair_cnt, part_o, part_ml, trace, total;
+      kv_len, tile_prefix, qscores, amax_val, amax_idx, pair_cnt, pad_cnt, part_o, part_ml, trace, total;
 };
 
 __host__ __device__ inline size_t ws_align(size_t x) { return (x + 255) & ~size_t(255); }
@@ -54,6 +54,8 @@ __host__ __device__ inline WsLayout ws_layout(int n_bs, int n_kv_heads, int num_
   L.amax_val = o;    o = ws_align(o + m_bs * kAccMaxChunks * 4);
   L.amax_idx = o;    o = ws_align(o + m_bs * kAccMaxChunks * 4);
   L.pair_cnt = o;    o = ws_align(o + size_t(n_bs) * n_kv_heads * 4);
+  // arrival counters of the padded comparison kernel: one per (request, q-head), group <= 8
+  L.pad_cnt = o;     o = ws_align(o + size_t(n_bs) * n_kv_heads * 8 * 4);
   // split-KV partials of the attention kernel: per CTA two slots (the segment
   // that starts its range and the one that ends it), each kTcRows rows of
   // (128 fp32 accumulators) plus (row max, row sum)

@@ -239,6 +239,27 @@ def test_attn_simt_other_group_sizes(P):
         _attn_parity(P, "simt", cfg)
 
 
+# ------------------------------------------------- padded comparison baseline
+@pytest.mark.parametrize("name,n_bs", [("tiny", 4), ("tiny", 6), ("qwen3_4b_layer", 8)])
+def test_padded_baseline_matches_unpacked_oracle(P, name, n_bs):
+    from oracle import verify_attn as OV
+    cfg = CONFIGS[name]
+    req, alloc, kc, vc, qu, qp = full_case(cfg, n_bs=n_bs)
+    ws = _ws(P, req)
+    st = StagedRequests(req)
+    gpu_alloc(P, ws, st)                                  # the baseline takes N from the workspace
+    out = torch.full(qu.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    P.verify_attn_padded(ws, qu.cuda(), kc.cuda(), vc.cuda(), st.block_table, st.ctx_len, SCALE, out)
+    torch.cuda.synchronize()
+    assert ws.status() == 0
+    ref = OV.verify_attn_padded(qu.float().numpy(), kc.float().numpy(), vc.float().numpy(),
+                                req["block_table"], req["ctx_len"], req["n_live"], cfg.n_q_heads,
+                                cfg.n_kv_heads, SCALE)
+    ok, max_abs, worst = attn_close(out, ref)
+    assert ok, f"padded: max|d|={max_abs} worst at {worst}"
+    assert (out[req["n_live"]:].float() == 0).all()
+
+
 # -------------------------------------------------------------- graph replay
 @pytest.mark.parametrize("impl", ["simt", "tensor"])
 def test_one_captured_graph_replays_at_any_mix_of_lengths(P, impl):
