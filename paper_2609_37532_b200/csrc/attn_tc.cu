@@ -206,6 +206,8 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     bool waited = false;       // griddepcontrol.wait done
     // lane l copies page l / 2, column half l % 2 (lanes 0..15)
     const int pg_l = lane >> 1, half = lane & 1;
+    // K/V are read exactly once per launch: mark them evict-first in L2
+    const uint64_t kv_policy = make_policy_evict_first();
     while (ok && sch.next(sg)) {
       const int qb = seg & 1;
       const int len = kv_len[sg.i];
@@ -229,8 +231,9 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           if (lane == 0) mbar_expect_tx(bar(B_KV_FULL + slot), n_pages * 2 * kPageBoxBytes);
           __syncwarp();
           if (lane < 16 && pg_l < n_pages) {
-            tma_load_5d(base + kOffKV + slot * kSlotBytes + half * kHalfSlot + pg_l * kPageBoxBytes,
-                        which == 0 ? &tm_k : &tm_v, bar(B_KV_FULL + slot), 0, half, 0, sg.g, page);
+            tma_load_5d_hint(base + kOffKV + slot * kSlotBytes + half * kHalfSlot + pg_l * kPageBoxBytes,
+                             which == 0 ? &tm_k : &tm_v, bar(B_KV_FULL + slot), 0, half, 0, sg.g, page,
+                             kv_policy);
           }
         }
         return true;
