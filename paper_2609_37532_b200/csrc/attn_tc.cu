@@ -60,7 +60,10 @@ namespace {
 
 constexpr int kThreads = 224;
 constexpr int kSoftmaxThreads = 128;
-constexpr int kStages = 5;
+#ifndef DSCALE_STAGES
+#define DSCALE_STAGES 5
+#endif
+constexpr int kStages = DSCALE_STAGES;
 constexpr int kSlotBytes = kTileTok * kD * 2;           // 32 KB: one K or V tile
 constexpr int kHalfSlot = kSlotBytes / 2;               // one 64-column half [128 tok][128 B]
 constexpr int kQBytes = kTcRows * kD * 2;               // 16 KB
@@ -238,6 +241,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         }
         return true;
       };
+      const int row0 = ws_ptr<int>(a.ws, L.offset)[sg.i];      // metadata: safe before the wait
       int t_first = sg.t0;
       if (!waited) {
         // before the grid dependency is resolved: up to two key tiles that lie wholly
@@ -257,7 +261,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       ok = mbar_wait(bar(B_Q_EMPTY + qb), ((seg >> 1) & 1) ^ 1, s_abort);
       if (!ok) break;
       if (lane == 0) {
-        const int row0 = ws_ptr<int>(a.ws, L.offset)[sg.i];
         mbar_expect_tx(bar(B_Q_FULL + qb), kQBytes);
         tma_load_4d(base + kOffQ + qb * kQBytes, &tm_q, bar(B_Q_FULL + qb), 0, 0, sg.g * 4, row0);
         tma_load_4d(base + kOffQ + qb * kQBytes + kQBytes / 2, &tm_q, bar(B_Q_FULL + qb), 0, 1,
@@ -885,7 +888,7 @@ bool kv_map(const void* ptr, int n_kv, int num_pages, CUtensorMap* out) {
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides,
                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   if (g_kv_maps.size() > 4096) g_kv_maps.clear();
   g_kv_maps[key] = *out;
