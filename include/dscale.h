@@ -262,6 +262,16 @@ int dscale_accept_static(int n_bs, const int32_t* n_live, const int32_t* k, cons
                          int32_t* out_len, void* stream);
 
 /*
+ * Bucket selection for a pool of captured capacities (Eq. 13):
+ * N_bs = min{ b in buckets : b >= n_live }.  HOST call.  Returns the chosen
+ * capacity, or DSCALE_ERR_TOO_LARGE if no bucket is large enough,
+ * DSCALE_ERR_INVALID_ARG for an empty / non-positive bucket set or n_live < 1.
+ * Each bucket has its own workspace and captured graph (Algorithm 2, lines 3-8);
+ * requests beyond n_live inside the chosen bucket are sentinels (Eq. 14).
+ */
+int dscale_select_bucket(const int32_t* buckets, int n_buckets, int n_live);
+
+/*
  * Device address of a workspace field (see DSCALE_WS_*), for tests and for
  * callers that feed packed fields to other kernels.  HOST call; returns NULL
  * for a bad field id.  The address depends only on (ws, n_bs).

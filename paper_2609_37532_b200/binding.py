@@ -46,6 +46,8 @@ lib.dscale_verify_attn_padded.restype = _i
 lib.dscale_verify_attn_padded.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i, _i, _vp, _i, _i, _f, _vp, _vp]
 lib.dscale_accept_static.restype = _i
 lib.dscale_accept_static.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _i64, _i, _vp, _vp, _vp, _vp, _vp]
+lib.dscale_select_bucket.restype = _i
+lib.dscale_select_bucket.argtypes = [_vp, _i, _i]
 lib.dscale_ws_field.restype = _vp
 lib.dscale_ws_field.argtypes = [_vp, _i, _i]
 lib.dscale_launches_per_call.restype = _i
@@ -234,3 +236,72 @@ def verify_attn_padded(ws, q_unpacked, k_cache, v_cache, block_table, ctx_len, s
                                          k_cache.shape[0], _ptr(ctx_len), ws.n_q_heads, ws.n_kv_heads,
                                          float(sm_scale), _ptr(out_unpacked), _stream()),
            "dscale_verify_attn_padded")
+
+
+class VerifyGraphPool:
+    """Fixed-address graph capture and replay over a set of request capacities
+    (Algorithm 2): one workspace, one set of fixed-address tensors and one
+    captured CUDA graph `[alloc -> attention x L -> accept]` per bucket; a step
+    picks the smallest bucket that holds the live requests (Eq. 13), writes its
+    inputs into that bucket's tensors and replays its graph.  Requests beyond N
+    in the bucket are sentinels.
+
+    The KV cache (one (k, v) pair per layer) is shared by all buckets; Q, logits
+    and outputs are per bucket because their shapes depend on the capacity."""
+
+    def __init__(self, buckets, n_q_heads: int, n_kv_heads: int, max_pages: int, kv_layers,
+                 vocab: int, sm_scale: float, device=None):
+        self.device = torch.device("cuda" if device is None else device)
+        self.buckets = sorted(int(b) for b in buckets)
+        self._barr = (C.c_int32 * len(self.buckets))(*self.buckets)
+        self.kv_layers, self.vocab, self.sm_scale = kv_layers, vocab, float(sm_scale)
+        self.max_pages, self.num_pages = max_pages, kv_layers[0][0].shape[0]
+        self.slots = {}
+        for b in self.buckets:
+            self.slots[b] = self._capture(b, n_q_heads, n_kv_heads)
+
+    def _capture(self, n_bs, n_q_heads, n_kv_heads):
+        dev, L = self.device, len(self.kv_layers)
+        i32 = dict(dtype=torch.int32, device=dev)
+        t = dict(
+            ws=VerifyWorkspace(n_bs, n_q_heads, n_kv_heads, device=dev),
+            n_live=torch.ones(1, **i32), scores=torch.zeros((n_bs, 15), dtype=torch.float32, device=dev),
+            draft=torch.zeros((n_bs, 16), **i32), ctx_len=torch.zeros(n_bs, **i32),
+            block_table=torch.zeros((n_bs, self.max_pages), **i32),
+            q=[torch.zeros((8 * n_bs, n_q_heads, 128), dtype=torch.bfloat16, device=dev) for _ in range(L)],
+            out=[torch.zeros((8 * n_bs, n_q_heads, 128), dtype=torch.bfloat16, device=dev) for _ in range(L)],
+            logits=torch.zeros((8 * n_bs, self.vocab), dtype=torch.float32, device=dev),
+            accept_len=torch.zeros(n_bs, **i32), next_anchor=torch.zeros(n_bs, **i32),
+            out_tokens=torch.zeros((n_bs, 16), **i32), out_len=torch.zeros(n_bs, **i32))
+
+        def step():
+            alloc_verify(t["ws"], t["n_live"], t["scores"], t["draft"], t["ctx_len"], t["block_table"],
+                         self.num_pages)
+            for l, (kc, vc) in enumerate(self.kv_layers):
+                verify_attn(t["ws"], t["q"][l], kc, vc, t["block_table"], self.sm_scale, t["out"][l])
+            accept(t["ws"], t["logits"], self.vocab, t["accept_len"], t["next_anchor"], t["out_tokens"],
+                   t["out_len"], None)
+
+        side = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(side):
+            step()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                step()
+        torch.cuda.synchronize()
+        t["graph"] = g
+        return t
+
+    def select(self, n_live: int) -> int:
+        b = lib.dscale_select_bucket(self._barr, len(self.buckets), int(n_live))
+        if b < 0:
+            raise DScaleError(b, "dscale_select_bucket")
+        return b
+
+    def slot(self, n_live: int):
+        """The fixed-address tensors of the bucket a batch of n_live requests uses."""
+        return self.slots[self.select(n_live)]
+
+    def replay(self, n_live: int):
+        self.slots[self.select(n_live)]["graph"].replay()

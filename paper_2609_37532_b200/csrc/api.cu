@@ -239,6 +239,16 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
   return DSCALE_OK;
 }
 
+int dscale_select_bucket(const int32_t* buckets, int n_buckets, int n_live) {
+  if (!buckets || n_buckets < 1 || n_live < 1) return DSCALE_ERR_INVALID_ARG;
+  int best = 0;
+  for (int b = 0; b < n_buckets; ++b) {
+    if (buckets[b] < 1) return DSCALE_ERR_INVALID_ARG;
+    if (buckets[b] >= n_live && (best == 0 || buckets[b] < best)) best = buckets[b];
+  }
+  return best ? best : DSCALE_ERR_TOO_LARGE;
+}
+
 const int32_t* dscale_ws_field(const void* ws, int n_bs, int field) {
   if (!ws || n_bs < 1 || n_bs > DSCALE_MAX_NBS) return nullptr;
   const WsLayout L = ws_layout(n_bs, 1, 1);      // index sections depend on n_bs only
