@@ -6,7 +6,7 @@ Greedy decoding (temperature 0): the target's token at a packed row is the
 index of the largest logit of that row, lowest index among equal maxima; a
 NaN never counts as a maximum.  Request i accepts its candidates in order
 while the target token predicted by the previous slot equals the candidate
-("Prefix verifier" paragraph): slot j's logits judge the token in slot j+1.
+("Prefix verifier" paragraph): slot j's logits decide on the token in slot j+1.
 After a_i accepted candidates the row offset_i + a_i supplies the successor,
 which is also the next anchor; if all k_i - 1 selected candidates pass, the
 last selected row supplies it.  Outputs follow Algorithm 2, lines 21-26:

@@ -736,7 +736,8 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     }
 #ifdef DSCALE_TRACE
     TRACE(60);
-    if (tid == 0) { trace[58] = wait_cycles; trace[59] = busy_cycles; trace[57] = it;
+    if (tid == 0) { unsigned smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid)); trace[51] = smid;
+                    trace[58] = wait_cycles; trace[59] = busy_cycles; trace[57] = it;
                     trace[52] = c_ld; trace[53] = c_max; trace[54] = c_pvw; trace[55] = c_exp; trace[56] = c_fence; }
 #endif
     // ---- end phase: publish what is left, merge the pairs this CTA is last to reach
