@@ -38,9 +38,9 @@
 //              it); it is only rescaled in place when a row maximum outgrows its
 //              reference by 2^8, and read back once per run for the epilogue.
 //   warp 6     publisher: fence + ticket for the first run's partial.
-// S is double-buffered in TMEM (2 x 128 columns) next to O (128 columns), P and
-// Q are double-buffered in shared memory, so the MMA of tile t+1 overlaps the
-// softmax of tile t.
+// S is triple-buffered in TMEM (3 x 128 columns) next to O (128 columns), P and
+// Q are double-buffered in shared memory; the MMA thread issues whichever of the
+// two products is ready, scores up to two tiles ahead of the softmax.
 //
 // Every wait is bounded: when a wait runs out the CTA sets the TIMEOUT status
 // bit, stops issuing work, drains its outstanding copies and releases TMEM.
@@ -75,7 +75,7 @@ constexpr int kOffQ = 0;                                 // 2 x 16 KB
 constexpr int kOffP = kOffQ + 2 * kQBytes;               // 2 x 16 KB
 constexpr int kOffKV = kOffP + 2 * kPBytes;              // 5 x 32 KB
 constexpr int kOffBar = kOffKV + kStages * kSlotBytes;   // mbarriers
-constexpr int kNumBars = 2 * kStages + 2 + 2 + 2 + 2 + 2 + 5;
+constexpr int kNumBars = 2 * kStages + 2 + 2 + 3 + 2 + 2 + 5;
 constexpr int kOffMisc = kOffBar + 8 * 32;               // tmem base, abort flag, tickets
 constexpr int kOffTile = kOffMisc + 48;                  // tile prefix, kMaxNbs + 1 ints
 constexpr int kSmemUse = kOffTile + (kMaxNbs + 1) * 4 + 12;
@@ -84,7 +84,7 @@ static_assert(kNumBars <= 32, "barrier area");
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
 
 enum Bar { B_KV_FULL = 0, B_KV_EMPTY = kStages, B_Q_FULL = 2 * kStages, B_Q_EMPTY = B_Q_FULL + 2,
-           B_S_FULL = B_Q_EMPTY + 2, B_P_FULL = B_S_FULL + 2, B_O_FULL = B_P_FULL + 2,
+           B_S_FULL = B_Q_EMPTY + 2, B_P_FULL = B_S_FULL + 3, B_O_FULL = B_P_FULL + 2,
            B_GROUP = B_O_FULL + 2,   // the 128 softmax threads among themselves
            B_PART = B_GROUP + 1,     // softmax -> publisher: the first run's partial is stored
            B_PUB = B_PART + 1,       // publisher -> softmax: that partial is published
@@ -152,9 +152,10 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     for (int s = 0; s < kStages; ++s) { mbar_init(bar(B_KV_FULL + s), 1); mbar_init(bar(B_KV_EMPTY + s), 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar(B_Q_FULL + b), 1); mbar_init(bar(B_Q_EMPTY + b), 1);
-      mbar_init(bar(B_S_FULL + b), 1); mbar_init(bar(B_P_FULL + b), kSoftmaxThreads);
+      mbar_init(bar(B_P_FULL + b), kSoftmaxThreads);
       mbar_init(bar(B_O_FULL + b), 1);
     }
+    for (int b = 0; b < 3; ++b) mbar_init(bar(B_S_FULL + b), 1);
     mbar_init(bar(B_GROUP), kSoftmaxThreads);
     mbar_init(bar(B_PART), kSoftmaxThreads);
     mbar_init(bar(B_PUB), 1);
@@ -346,60 +347,84 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   } else if (warp == 7) {
 #endif
     if (lane == 0) {
+      // Event-driven issue.  S = Q K^T of tile x goes into TMEM buffer x % 3 as soon
+      // as its K slot has landed and that buffer's previous tile (x - 3) has been
+      // read by the softmax warps; O += P V of tile y as soon as P_y and V_y are
+      // there.  Scores may run up to two tiles ahead of the softmax, which frees K
+      // slots early and keeps more page copies in flight.
       Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
       Segment sg;
-      unsigned it = 0;
-      int seg = 0;
+      const unsigned total = (unsigned)(sl_end - sl_begin);
+      unsigned next_s = 0, next_pv = 0;
+      int seg = -1, t = 0, t_end = 0;            // S cursor: current run and tile inside it
+      bool q_ready = false;
+      unsigned run_start_mask = 0;               // bit (x % 4): tile x starts a run
       bool ok = true;
-      bool first_of_run[2] = {true, true};   // per P buffer: does its tile start a run?
-      auto issue_pv = [&](unsigned pt) -> bool {
-        const int b = pt & 1;
-        const unsigned uv = 2 * pt + 1;
-        const int slot = uv % kStages;
-        if (!mbar_wait(bar(B_P_FULL + b), (pt >> 1) & 1, s_abort)) return false;
-        if (!mbar_wait(bar(B_KV_FULL + slot), (uv / kStages) & 1, s_abort)) return false;
-        tc_fence_after();
-        const uint32_t p_base = base + kOffP + b * kPBytes;
-        const uint32_t v_base = base + kOffKV + slot * kSlotBytes;
+      long long t_idle = clock64();
+      while (ok && next_pv < total) {
+        bool progressed = false;
+        // ---- O += P V for the oldest tile whose P is ready
+        if (next_pv < next_s) {
+          const unsigned pt = next_pv;
+          const int b = pt & 1;
+          const unsigned uv = 2 * pt + 1;
+          const int slot = uv % kStages;
+          if (mbar_try(bar(B_P_FULL + b), (pt >> 1) & 1) && mbar_try(bar(B_KV_FULL + slot), (uv / kStages) & 1)) {
+            tc_fence_after();
+            const uint32_t p_base = base + kOffP + b * kPBytes;
+            const uint32_t v_base = base + kOffKV + slot * kSlotBytes;
+            const bool fresh = (run_start_mask >> (pt & 3)) & 1;
 #pragma unroll
-        for (int kk = 0; kk < kTileTok / 16; ++kk) {
-          // A = P [64 rows][128 tok] K-major: 64-token blocks of 8 KB, 32 B per 16 tokens
-          const uint64_t ad = smem_desc(p_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
-          // B = V [128 tok][128 d] with d contiguous: MN-major, 16 tokens = 2 KB
-          const uint64_t bd = smem_desc(v_base + kk * (16 * 128), kHalfSlot, 1024);
-          umma(tmem + 256, ad, bd, kIdescPV, (kk > 0) || !first_of_run[b]);
-        }
-        umma_commit(bar(B_O_FULL + b));
-        umma_commit(bar(B_KV_EMPTY + slot));
-        return true;
-      };
-      while (ok && sch.next(sg)) {
-        const int qb = seg & 1;
-        ok = mbar_wait(bar(B_Q_FULL + qb), (seg >> 1) & 1, s_abort);
-        for (int t = sg.t0; t < sg.t1 && ok; ++t, ++it) {
-          const int b = it & 1;
-          first_of_run[b] = (t == sg.t0);
-          const unsigned uk = 2 * it;
-          const int slot = uk % kStages;
-          ok = mbar_wait(bar(B_KV_FULL + slot), (uk / kStages) & 1, s_abort);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t q_base = base + kOffQ + qb * kQBytes;
-          const uint32_t k_base = base + kOffKV + slot * kSlotBytes;
-#pragma unroll
-          for (int kk = 0; kk < kD / 16; ++kk) {
-            const uint64_t ad = smem_desc(q_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
-            const uint64_t bd = smem_desc(k_base + (kk >> 2) * kHalfSlot + (kk & 3) * 32, 16, 1024);
-            umma(tmem + b * 128, ad, bd, kIdescS, kk > 0);
+            for (int kk = 0; kk < kTileTok / 16; ++kk) {
+              // A = P [64 rows][128 tok] K-major: 64-token blocks of 8 KB, 32 B per 16 tokens
+              const uint64_t ad = smem_desc(p_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
+              // B = V [128 tok][128 d] with d contiguous: MN-major, 16 tokens = 2 KB
+              const uint64_t bd = smem_desc(v_base + kk * (16 * 128), kHalfSlot, 1024);
+              umma(tmem + 384, ad, bd, kIdescPV, (kk > 0) || !fresh);
+            }
+            umma_commit(bar(B_O_FULL + b));
+            umma_commit(bar(B_KV_EMPTY + slot));
+            ++next_pv;
+            progressed = true;
           }
-          umma_commit(bar(B_S_FULL + b));
-          umma_commit(bar(B_KV_EMPTY + slot));
-          if (t + 1 == sg.t1) umma_commit(bar(B_Q_EMPTY + qb));
-          if (it >= 1) ok = issue_pv(it - 1);
         }
-        ++seg;
+        // ---- S = Q K^T for the next tile, at most two tiles ahead of the P V cursor
+        if (next_s < total && next_s <= next_pv + 2) {
+          if (t == t_end) {                         // next run
+            sch.next(sg);
+            ++seg; t = sg.t0; t_end = sg.t1; q_ready = false;
+          }
+          const int qb = seg & 1;
+          if (!q_ready) q_ready = mbar_try(bar(B_Q_FULL + qb), (seg >> 1) & 1);
+          const unsigned uk = 2 * next_s;
+          const int slot = uk % kStages;
+          if (q_ready && mbar_try(bar(B_KV_FULL + slot), (uk / kStages) & 1)) {
+            tc_fence_after();
+            const int b3 = next_s % 3;
+            const uint32_t q_base = base + kOffQ + qb * kQBytes;
+            const uint32_t k_base = base + kOffKV + slot * kSlotBytes;
+#pragma unroll
+            for (int kk = 0; kk < kD / 16; ++kk) {
+              const uint64_t ad = smem_desc(q_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
+              const uint64_t bd = smem_desc(k_base + (kk >> 2) * kHalfSlot + (kk & 3) * 32, 16, 1024);
+              umma(tmem + b3 * 128, ad, bd, kIdescS, kk > 0);
+            }
+            umma_commit(bar(B_S_FULL + b3));
+            umma_commit(bar(B_KV_EMPTY + slot));
+            if (t + 1 == t_end) umma_commit(bar(B_Q_EMPTY + qb));
+            run_start_mask = (run_start_mask & ~(1u << (next_s & 3))) | ((t == sg.t0 ? 1u : 0u) << (next_s & 3));
+            ++t;
+            ++next_s;
+            progressed = true;
+          }
+        }
+        if (progressed) {
+          t_idle = clock64();
+        } else {
+          if (*s_abort) ok = false;
+          else if (clock64() - t_idle > kWaitCycles) { *s_abort = 1; ok = false; }
+        }
       }
-      if (ok && it >= 1) ok = issue_pv(it - 1);
     }
     __syncwarp();
   } else if (warp == 6) {
@@ -454,7 +479,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     const int quad = lane & 3;
     const int rowv[2] = {warp * 16 + (lane >> 2), warp * 16 + (lane >> 2) + 8};
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
-    const uint32_t o_addr = t_lane + 256;
+    const uint32_t o_addr = t_lane + 384;
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
     float* part_o = ws_ptr<float>(a.ws, L.part_o);
     float* part_ml = ws_ptr<float>(a.ws, L.part_ml);
@@ -530,7 +555,8 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 #ifdef DSCALE_TRACE
         const long long tw0 = clock64();
 #endif
-        ok = mbar_wait(bar(B_S_FULL + b), (it >> 1) & 1, s_abort);
+        const int b3 = it % 3;                   // the three score buffers in TMEM
+        ok = mbar_wait(bar(B_S_FULL + b3), (it / 3) & 1, s_abort);
         if (!ok) break;
         tc_fence_after();
 #ifdef DSCALE_TRACE
@@ -539,7 +565,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         wait_cycles += tw1 - tw0;
 #endif
         float s[64];
-        tmem_ld_16x128(t_lane + b * 128, s);
+        tmem_ld_16x128(t_lane + b3 * 128, s);
 #ifdef DSCALE_TRACE
         const long long tw2 = clock64();
         c_ld += tw2 - tw1;
