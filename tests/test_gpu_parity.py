@@ -233,6 +233,22 @@ def test_attn_skewed_lengths(P, impl):
     _attn_parity(P, impl, cfg, n_bs=8)
 
 
+@pytest.mark.parametrize("impl", ["simt", "tensor"])
+def test_attn_pairs_cut_across_many_ctas(P, impl):
+    # two long requests on two kv-heads: every (request, kv-head) pair spans dozens of CTAs of the
+    # persistent grid, so the split-KV merge sees many contributors per pair
+    cfg = small_variant(CONFIGS["tiny"], n=2, seed=41)
+    _attn_parity(P, impl, cfg, ctx_override=[20000, 9000])
+
+
+@pytest.mark.parametrize("impl", ["simt", "tensor"])
+def test_attn_full_capacity_of_64_requests(P, impl):
+    cfg = small_variant(CONFIGS["tiny"], n=64, seed=43, ctx_lo=0, ctx_hi=300)
+    _attn_parity(P, impl, cfg)
+    cfg = small_variant(CONFIGS["tiny"], n=37, seed=44, ctx_lo=100, ctx_hi=900)
+    _attn_parity(P, impl, cfg, n_bs=64)
+
+
 def test_attn_simt_other_group_sizes(P):
     for hq, hkv in ((4, 4), (8, 4), (8, 1)):
         cfg = small_variant(CONFIGS["tiny"], n_q_heads=hq, n_kv_heads=hkv, seed=21)
