@@ -327,6 +327,17 @@ def run_ours(args, rank, world, local_rank):
         eb.record(stream)
         barrier()
         accept_ms = ea.elapsed_time(eb) / args.steps
+        # the sampling verifier (temperature 1) on the same logits, for its own figure
+        u_acc = torch.rand(8 * n_bs, device=dev)
+        u_drw = torch.rand(n_bs, device=dev)
+        so = [torch.zeros_like(outs[0]), torch.zeros_like(outs[1]), torch.zeros_like(outs[2]), torch.zeros_like(outs[3])]
+        P.accept_sampling(ws, logits, cfg.vocab, 1.0, u_acc, u_drw, so[0], so[1], so[2], so[3])
+        ea.record(stream)
+        for _ in range(args.steps):
+            P.accept_sampling(ws, logits, cfg.vocab, 1.0, u_acc, u_drw, so[0], so[1], so[2], so[3])
+        eb.record(stream)
+        barrier()
+        sampling_ms = ea.elapsed_time(eb) / args.steps
 
         # ---- timed region 3: end to end through the host-buffer C ABI call ----
         hs = P.HostStep(ws, req["max_pages"], req["num_pages"], layers, logits, cfg.vocab, SCALE)
@@ -379,7 +390,7 @@ def run_ours(args, rank, world, local_rank):
                          "frac": achieved / peak, "frac_of_8tbs": achieved / 8000.0,
                          "bytes_per_launch": per_layer_b, "us_per_launch": attn_ms * 1e3,
                          "traffic": recorded_traffic(cfg.name)},
-            "accept_us": accept_ms * 1e3,
+            "accept_us": accept_ms * 1e3, "accept_sampling_us": sampling_ms * 1e3,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": hs.h2d_bytes,
                     "d2h_bytes_per_step": hs.d2h_bytes, "ms_per_step": 1e3 * e2e_s / args.steps,
                     "api": "dscale_verify_step_host (pinned host inputs/outputs, KV/Q/logits resident)"},

@@ -233,6 +233,30 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
                             int32_t* h_out_tokens, int32_t* h_out_len, void* stream);
 
 /*
+ * Prefix verification under a sampling target policy ("Prefix verifier"
+ * paragraph, temperature > 0).  P = softmax(logits / temperature) at each packed
+ * row.  The candidate x in slot j + 1 is accepted iff u_accept[offset_i + j] < P(x);
+ * at the first rejection the successor is drawn from P with x removed and the
+ * rest renormalised, and if all k_i - 1 selected candidates pass it is drawn
+ * from the unmodified P of the last selected row.  The draw is the first index
+ * whose cumulative weight exceeds u_draw[i] times the total (inverse CDF in
+ * index order).  Random numbers are inputs, so the lengths do not depend on them
+ * and a replayed graph only needs fresh uniforms at the same addresses.
+ *
+ *   u_accept  fp32 [8 n_bs], one uniform in [0,1) per packed row
+ *   u_draw    fp32 [n_bs],   one uniform in [0,1) per request
+ *   p_draft   nullable fp32 [8 n_bs]: receives P(candidate) of every row that has one
+ *   outputs   as in dscale_accept
+ * Logits must be finite.  Probabilities are evaluated in fp32; a draw whose
+ * target falls within rounding of a boundary of the cumulative sum may return
+ * the neighbouring token.
+ */
+int dscale_accept_sampling(void* ws, int n_bs, const float* logits, int64_t ld, int vocab,
+                           float temperature, const float* u_accept, const float* u_draw,
+                           int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
+                           int32_t* out_len, float* p_draft, void* stream);
+
+/*
  * Greedy prefix verification for callers that can neither allocate nor keep a
  * workspace.  (The paper has no counterpart to this call: it exists for
  * deployment reasons only.)  Typical users: a serving loop in which a cudaMalloc
@@ -279,7 +303,8 @@ int dscale_select_bucket(const int32_t* buckets, int n_buckets, int n_live);
 const int32_t* dscale_ws_field(const void* ws, int n_bs, int field);
 
 /* Number of kernels the three stage calls enqueue (for launch accounting):
- * which = 0 alloc, 1 attention, 2 accept, 3 attention (simt), 4 attention (padded). */
+ * which = 0 alloc, 1 attention, 2 accept, 3 attention (simt), 4 attention (padded),
+ * 5 accept (sampling). */
 int dscale_launches_per_call(int which);
 
 #ifdef __cplusplus

@@ -46,6 +46,8 @@ lib.dscale_verify_attn_padded.restype = _i
 lib.dscale_verify_attn_padded.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i, _i, _vp, _i, _i, _f, _vp, _vp]
 lib.dscale_accept_static.restype = _i
 lib.dscale_accept_static.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _i64, _i, _vp, _vp, _vp, _vp, _vp]
+lib.dscale_accept_sampling.restype = _i
+lib.dscale_accept_sampling.argtypes = [_vp, _i, _vp, _i64, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.dscale_select_bucket.restype = _i
 lib.dscale_select_bucket.argtypes = [_vp, _i, _i]
 lib.dscale_ws_field.restype = _vp
@@ -305,3 +307,18 @@ class VerifyGraphPool:
 
     def replay(self, n_live: int):
         self.slots[self.select(n_live)]["graph"].replay()
+
+
+def accept_sampling(ws, logits, vocab: int, temperature: float, u_accept, u_draw, accept_len,
+                    next_anchor, out_tokens, out_len, p_draft=None):
+    """Prefix verification under a sampling target policy (dscale_accept_sampling)."""
+    _need(logits, torch.float32, "logits"); _need(u_accept, torch.float32, "u_accept")
+    _need(u_draw, torch.float32, "u_draw")
+    for n, t in (("accept_len", accept_len), ("next_anchor", next_anchor),
+                 ("out_tokens", out_tokens), ("out_len", out_len)):
+        _need(t, torch.int32, n)
+    assert u_accept.shape == (8 * ws.n_bs,) and u_draw.shape == (ws.n_bs,)
+    _check(lib.dscale_accept_sampling(C.c_void_p(ws.ptr), ws.n_bs, _ptr(logits), logits.stride(0), vocab,
+                                      float(temperature), _ptr(u_accept), _ptr(u_draw), _ptr(accept_len),
+                                      _ptr(next_anchor), _ptr(out_tokens), _ptr(out_len), _ptr(p_draft),
+                                      _stream()), "dscale_accept_sampling")

@@ -239,6 +239,21 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
   return DSCALE_OK;
 }
 
+int dscale_accept_sampling(void* ws, int n_bs, const float* logits, int64_t ld, int vocab,
+                           float temperature, const float* u_accept, const float* u_draw,
+                           int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
+                           int32_t* out_len, float* p_draft, void* stream) {
+  if (!ws || !logits || !u_accept || !u_draw || !accept_len || !next_anchor || !out_tokens || !out_len)
+    return DSCALE_ERR_INVALID_ARG;
+  if (vocab < 1 || ld < vocab || (ld % 4) != 0 || !aligned(logits, 16) || !(temperature > 0.0f))
+    return DSCALE_ERR_INVALID_ARG;
+  WsInfo info;
+  if (!lookup(ws, n_bs, &info)) return DSCALE_ERR_WORKSPACE;
+  SampleArgs a{ws, n_bs, logits, ld, vocab, temperature, u_accept, u_draw, accept_len, next_anchor,
+               out_tokens, out_len, p_draft, info.n_kv_heads, info.num_ctas};
+  return launch_accept_sampling(a, (cudaStream_t)stream) == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
+}
+
 int dscale_select_bucket(const int32_t* buckets, int n_buckets, int n_live) {
   if (!buckets || n_buckets < 1 || n_live < 1) return DSCALE_ERR_INVALID_ARG;
   int best = 0;
@@ -278,6 +293,7 @@ int dscale_launches_per_call(int which) {
     case 2: return 1;   // accept_kernel
     case 3: return 1;   // attn_simt_kernel
     case 4: return 1;   // attn_padded_kernel
+    case 5: return 2;   // sample_stats_kernel + sample_draw_kernel
     default: return 0;
   }
 }

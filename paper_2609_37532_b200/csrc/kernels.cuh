@@ -58,6 +58,25 @@ cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t stream);
 // returns cudaErrorNotSupported if the driver entry point for tensor maps is missing
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t stream);
 
+struct SampleArgs {
+  void* ws;
+  int n_bs;
+  const float* logits;
+  int64_t ld;
+  int vocab;
+  float temperature;
+  const float* u_accept;   // [8 n_bs] one uniform per packed row
+  const float* u_draw;     // [n_bs]   one uniform per request
+  int32_t* accept_len;
+  int32_t* next_anchor;
+  int32_t* out_tokens;
+  int32_t* out_len;
+  float* p_draft;          // nullable [8 n_bs]: P(candidate) per row
+  int n_kv_heads;
+  int num_ctas;
+};
+cudaError_t launch_accept_sampling(const SampleArgs& a, cudaStream_t stream);
+
 // comparison baseline: unpacked W = 16, one 128-row tile per (request, q-head)
 cudaError_t launch_attn_padded(void* ws, int n_bs, const void* q_unpacked, const void* k_cache,
                                const void* v_cache, const int32_t* block_table, int max_pages,

@@ -23,12 +23,13 @@ constexpr int kTcRows = 64;       // rows of the tensor-core query tile (GQA gro
 // header words (int32)
 enum HdrWord {
   H_STATUS = 0, H_N_LIVE = 1, H_M_LIVE = 2, H_TOTAL_TILES = 3, H_ACCEPT_TICKET = 4,
-  H_MAGIC = 5, H_WORDS = 64
+  H_MAGIC = 5, H_SAMPLE_TICKET = 6, H_WORDS = 64
 };
 
 struct WsLayout {
   size_t hdr, k, k0, offset, q_start, q_end, tokens, positions, kv_refs, row_req, top1,
-      kv_len, tile_prefix, qscores, amax_val, amax_idx, pair_cnt, pad_cnt, part_o, part_ml, trace, total;
+      kv_len, tile_prefix, qscores, amax_val, amax_idx, smp_m, smp_s, row_m, row_z, row_flag, req_row, req_rej, pair_cnt, pad_cnt,
+      part_o, part_ml, trace, total;
 };
 
 __host__ __device__ inline size_t ws_align(size_t x) { return (x + 255) & ~size_t(255); }
@@ -53,6 +54,15 @@ __host__ __device__ inline WsLayout ws_layout(int n_bs, int n_kv_heads, int num_
   L.qscores = o;     o = ws_align(o + size_t(n_bs) * kW * 4);
   L.amax_val = o;    o = ws_align(o + m_bs * kAccMaxChunks * 4);
   L.amax_idx = o;    o = ws_align(o + m_bs * kAccMaxChunks * 4);
+  // sampling verifier: per (row, chunk) running (max, sum), per-row totals and
+  // acceptance flags, per-request row that supplies the successor
+  L.smp_m = o;       o = ws_align(o + m_bs * kAccMaxChunks * 4);
+  L.smp_s = o;       o = ws_align(o + m_bs * kAccMaxChunks * 4);
+  L.row_m = o;       o = ws_align(o + m_bs * 4);
+  L.row_z = o;       o = ws_align(o + m_bs * 4);
+  L.row_flag = o;    o = ws_align(o + m_bs * 4);
+  L.req_row = o;     o = ws_align(o + n_bs * 4);
+  L.req_rej = o;     o = ws_align(o + n_bs * 4);
   L.pair_cnt = o;    o = ws_align(o + size_t(n_bs) * n_kv_heads * 4);
   // arrival counters of the padded comparison kernel: one per (request, q-head), group <= 8
   L.pad_cnt = o;     o = ws_align(o + size_t(n_bs) * n_kv_heads * 8 * 4);
