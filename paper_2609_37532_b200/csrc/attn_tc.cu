@@ -273,7 +273,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         if (t + 1 < sg.t1) page_next = fetch_page(t + 1);
         ok = issue_tile(t, page);
       }
-#ifndef DSCALE_STREAM_ONLY
       if (ok && run_kind(sg, sch.more()) == RUN_TAIL) {
         // The slice ends inside this pair.  If every other contributor has already
         // published its partial (the usual case: they computed theirs at the start
@@ -310,7 +309,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         __syncwarp();
         if (lane == 0) { *s_fast = ok ? fast : 0; mbar_arrive(bar(B_PARTNER)); }
       }
-#endif
       ++seg;
     }
     if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -322,30 +320,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     }
   } else if (warp == 5) {
     // ============================================================ MMA issuer
-#ifdef DSCALE_STREAM_ONLY
-    // probe build: consume every K/V slot as soon as it lands, no math at all;
-    // measures what the TMA page stream alone can sustain
-    if (lane == 0) {
-      Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
-      Segment sg;
-      unsigned u = 0;
-      int seg = 0;
-      bool ok = true;
-      while (ok && sch.next(sg)) {
-        ok = mbar_wait(bar(B_Q_FULL + (seg & 1)), (seg >> 1) & 1, s_abort);
-        for (int t = sg.t0; t < sg.t1 && ok; ++t) {
-          for (int which = 0; which < 2 && ok; ++which, ++u) {
-            ok = mbar_wait(bar(B_KV_FULL + u % kStages), (u / kStages) & 1, s_abort);
-            mbar_arrive(bar(B_KV_EMPTY + u % kStages));
-          }
-        }
-        mbar_arrive(bar(B_Q_EMPTY + (seg & 1)));
-        ++seg;
-      }
-    }
-    __syncwarp();
-  } else if (warp == 7) {
-#endif
     if (lane == 0) {
       // Event-driven issue.  S = Q K^T of tile x goes into TMEM buffer x % 3 as soon
       // as its K slot has landed and that buffer's previous tile (x - 3) has been
@@ -435,11 +409,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     // microseconds while the SM streams; here they delay nobody.
     Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
     Segment sg;
-#ifdef DSCALE_STREAM_ONLY
-    if (false) {
-#else
     if (sch.next(sg) && run_kind(sg, sch.more()) == RUN_PUBLISH) {
-#endif
       if (mbar_wait(bar(B_PART), 0, s_abort)) {
         __threadfence();
         if (lane == 0) {
@@ -454,13 +424,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       }
     }
     __syncwarp();
-#ifdef DSCALE_STREAM_ONLY
-  } else if (warp < 4) {
-    // probe build: no softmax, no output
-  } else if (warp == 8) {
-#else
   } else {
-#endif
     // ====================================================== softmax warps 0-3
     // rows of capacity beyond M_live are written as zero, spread over the grid
     {
