@@ -27,8 +27,8 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from dscale_inputs import (CONFIGS, make_kv_layer, make_logits_unpacked, make_q_unpacked,  # noqa: E402
-                           make_requests, rows_to_packed, small_variant)
+from dscale_inputs import (CONFIGS, make_kv_layer, make_lm_head_unpacked, make_logits_unpacked,  # noqa: E402
+                           make_q_unpacked, make_requests, rows_to_packed, small_variant)
 
 SCALE = 1.0 / float(np.sqrt(128.0))
 METRIC = "verified_tokens_per_s"
@@ -339,6 +339,37 @@ def run_ours(args, rank, world, local_rank):
         barrier()
         sampling_ms = ea.elapsed_time(eb) / args.steps
 
+        # the fused LM head + argmax + acceptance (one launch) on seeded hidden states
+        lm = None
+        if args.lm_hidden > 0:
+            w_lm, h_un = make_lm_head_unpacked(req, args.lm_hidden, device=str(dev))
+            h_lm = rows_to_packed(h_un, k, offset, n, 8 * n_bs)
+            del h_un
+            lo = [torch.zeros_like(x) for x in outs[:4]]
+            for _ in range(3):
+                P.lm_head_accept(ws, h_lm, w_lm, lo[0], lo[1], lo[2], lo[3])
+            ea.record(stream)
+            for _ in range(args.steps):
+                P.lm_head_accept(ws, h_lm, w_lm, lo[0], lo[1], lo[2], lo[3])
+            eb.record(stream)
+            barrier()
+            lm_ms = ea.elapsed_time(eb) / args.steps
+            # context: the library GEMM that would only produce the logits (bf16 out)
+            for _ in range(2):
+                lg = torch.matmul(h_lm, w_lm.t())
+            ea.record(stream)
+            for _ in range(args.steps):
+                lg = torch.matmul(h_lm, w_lm.t())
+            eb.record(stream)
+            barrier()
+            gemm_ms = ea.elapsed_time(eb) / args.steps
+            lm_bytes = w_lm.numel() * 2 + h_lm.numel() * 2
+            lm_flops = 2.0 * 8 * n * cfg.vocab * args.lm_hidden
+            lm = {"us": lm_ms * 1e3, "hidden": args.lm_hidden, "bytes": lm_bytes,
+                  "gbs": lm_bytes / (lm_ms * 1e-3) / 1e9, "tflops": lm_flops / (lm_ms * 1e-3) / 1e12,
+                  "library_gemm_logits_only_us": gemm_ms * 1e3}
+            del w_lm, h_lm, lg
+
         # ---- timed region 3: end to end through the host-buffer C ABI call ----
         hs = P.HostStep(ws, req["max_pages"], req["num_pages"], layers, logits, cfg.vocab, SCALE)
         hs.h_n_live[0] = n
@@ -391,6 +422,7 @@ def run_ours(args, rank, world, local_rank):
                          "bytes_per_launch": per_layer_b, "us_per_launch": attn_ms * 1e3,
                          "traffic": recorded_traffic(cfg.name)},
             "accept_us": accept_ms * 1e3, "accept_sampling_us": sampling_ms * 1e3,
+            "lm_head_accept": lm,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": hs.h2d_bytes,
                     "d2h_bytes_per_step": hs.d2h_bytes, "ms_per_step": 1e3 * e2e_s / args.steps,
                     "api": "dscale_verify_step_host (pinned host inputs/outputs, KV/Q/logits resident)"},
@@ -445,6 +477,8 @@ def main():
     ap.add_argument("--workload", default="qwen3_8b_step", choices=list(CONFIGS))
     ap.add_argument("--attn", default="tensor", choices=["tensor", "simt"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
+    ap.add_argument("--lm-hidden", type=int, default=4096,
+                    help="hidden size of the fused LM-head figure (0 skips it)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-padded", action="store_true", help="skip the padded comparison kernel")
     ap.add_argument("--cpu-layers", type=int, default=0,

@@ -198,6 +198,31 @@ def make_logits_unpacked(req: dict, device: str = "cpu") -> torch.Tensor:
     return logits
 
 
+def make_lm_head_unpacked(req: dict, hidden_dim: int, device: str = "cpu"):
+    """Inputs of the LM head: (weight bf16 [vocab, hidden_dim], hidden bf16
+    [n_bs, W, hidden_dim]).  Weights are N(0,1); every slot's final hidden
+    state is N(0, 0.25 / hidden_dim) noise (logits of standard deviation
+    0.5), and the slots that carry the planted acceptance (the same ones
+    make_logits_unpacked boosts) additionally point
+    along the weight row of their planted token, scaled so that token's logit
+    is about 8 while all others stay below about 3."""
+    cfg = req["cfg"]
+    g = torch.Generator(device=device)
+    g.manual_seed(cfg.seed * 1_000_003 + 130363)
+    n_bs = req["n_bs"]
+    weight = torch.randn((cfg.vocab, hidden_dim), generator=g, dtype=torch.float32,
+                         device=device).to(torch.bfloat16)
+    hidden = (0.5 / hidden_dim ** 0.5) * torch.randn((n_bs, W, hidden_dim), generator=g, dtype=torch.float32, device=device)
+    draft = req["draft_tokens"]
+    for i in range(req["n_live"]):
+        a = int(req["planted_a"][i])
+        for j in range(a + 1):
+            tok = int(draft[i, j + 1]) if j < a else int(req["planted_next"][i])
+            w = weight[tok].float()
+            hidden[i, j] += 8.0 * w / float(w @ w)
+    return weight, hidden.to(torch.bfloat16)
+
+
 def rows_to_packed(unpacked: torch.Tensor, k, offset, n_live: int, m_bs: int,
                    fill: float = 0.0) -> torch.Tensor:
     """Lay the first k_i slot rows of each request at rows offset_i .. of a

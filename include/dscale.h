@@ -233,6 +233,24 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
                             int32_t* h_out_tokens, int32_t* h_out_len, void* stream);
 
 /*
+ * Fused LM head + greedy prefix verification: dscale_accept without the logits.
+ * The target token of packed row s is argmax_v sum_h hidden[s][h] * weight[v][h]
+ * (the LM head applied to the M = 8N packed rows DVL leaves, Section 3.3), computed
+ * on the tensor cores tile by tile with a running (max, first index) per row, so
+ * the 8N x V logits are never written; then the same acceptance loop and outputs
+ * as dscale_accept (Algorithm 2, lines 21-26).
+ *
+ *   hidden   bf16 [8 n_bs][hidden_dim], packed rows, hidden_dim % 64 == 0
+ *   weight   bf16 [vocab][hidden_dim] (one row per vocabulary entry), vocab >= 16
+ *   row_max  nullable fp32 [8 n_bs]: receives the winning logit of every live row
+ * Products are accumulated in fp32; two logits closer than fp32 rounding of the
+ * dot product may resolve differently from an exact evaluation.
+ */
+int dscale_lm_head_accept(void* ws, int n_bs, const void* hidden, const void* weight, int hidden_dim,
+                          int vocab, int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
+                          int32_t* out_len, int32_t* ctx_len_inout, float* row_max, void* stream);
+
+/*
  * Prefix verification under a sampling target policy ("Prefix verifier"
  * paragraph, temperature > 0).  P = softmax(logits / temperature) at each packed
  * row.  The candidate x in slot j + 1 is accepted iff u_accept[offset_i + j] < P(x);
@@ -304,7 +322,7 @@ const int32_t* dscale_ws_field(const void* ws, int n_bs, int field);
 
 /* Number of kernels the three stage calls enqueue (for launch accounting):
  * which = 0 alloc, 1 attention, 2 accept, 3 attention (simt), 4 attention (padded),
- * 5 accept (sampling). */
+ * 5 accept (sampling), 6 fused LM head + accept. */
 int dscale_launches_per_call(int which);
 
 #ifdef __cplusplus

@@ -46,6 +46,8 @@ lib.dscale_verify_attn_padded.restype = _i
 lib.dscale_verify_attn_padded.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i, _i, _vp, _i, _i, _f, _vp, _vp]
 lib.dscale_accept_static.restype = _i
 lib.dscale_accept_static.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _i64, _i, _vp, _vp, _vp, _vp, _vp]
+lib.dscale_lm_head_accept.restype = _i
+lib.dscale_lm_head_accept.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.dscale_accept_sampling.restype = _i
 lib.dscale_accept_sampling.argtypes = [_vp, _i, _vp, _i64, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.dscale_select_bucket.restype = _i
@@ -322,3 +324,17 @@ def accept_sampling(ws, logits, vocab: int, temperature: float, u_accept, u_draw
                                       float(temperature), _ptr(u_accept), _ptr(u_draw), _ptr(accept_len),
                                       _ptr(next_anchor), _ptr(out_tokens), _ptr(out_len), _ptr(p_draft),
                                       _stream()), "dscale_accept_sampling")
+
+
+def lm_head_accept(ws, hidden, weight, accept_len, next_anchor, out_tokens, out_len,
+                   ctx_len_inout=None, row_max=None):
+    """Fused LM head + argmax + greedy acceptance (dscale_lm_head_accept)."""
+    _need(hidden, torch.bfloat16, "hidden"); _need(weight, torch.bfloat16, "weight")
+    for n, t in (("accept_len", accept_len), ("next_anchor", next_anchor),
+                 ("out_tokens", out_tokens), ("out_len", out_len)):
+        _need(t, torch.int32, n)
+    assert hidden.shape[0] == 8 * ws.n_bs and hidden.shape[1] == weight.shape[1]
+    _check(lib.dscale_lm_head_accept(C.c_void_p(ws.ptr), ws.n_bs, _ptr(hidden), _ptr(weight), hidden.shape[1],
+                                     weight.shape[0], _ptr(accept_len), _ptr(next_anchor), _ptr(out_tokens),
+                                     _ptr(out_len), _ptr(ctx_len_inout), _ptr(row_max), _stream()),
+           "dscale_lm_head_accept")

@@ -12,6 +12,7 @@ namespace dscale {
 cudaError_t attn_simt_prepare();
 cudaError_t attn_tc_prepare();
 cudaError_t attn_padded_prepare();
+cudaError_t lm_head_prepare();
 }
 
 namespace {
@@ -66,6 +67,7 @@ int dscale_workspace_init(void* ws, size_t bytes, int n_bs, int n_q_heads, int n
   if (attn_simt_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
   if (attn_tc_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
   if (attn_padded_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
+  if (lm_head_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
   std::lock_guard<std::mutex> lk(g_mu);
   g_ws[ws] = WsInfo{bytes, n_bs, n_q_heads, n_kv_heads, num_sms};
   return DSCALE_OK;
@@ -239,6 +241,22 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
   return DSCALE_OK;
 }
 
+int dscale_lm_head_accept(void* ws, int n_bs, const void* hidden, const void* weight, int hidden_dim,
+                          int vocab, int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
+                          int32_t* out_len, int32_t* ctx_len_inout, float* row_max, void* stream) {
+  if (!ws || !hidden || !weight || !accept_len || !next_anchor || !out_tokens || !out_len)
+    return DSCALE_ERR_INVALID_ARG;
+  if (!aligned(hidden, 16) || !aligned(weight, 16)) return DSCALE_ERR_INVALID_ARG;
+  if (hidden_dim < 64 || hidden_dim % 64 != 0 || vocab < 16) return DSCALE_ERR_UNSUPPORTED;
+  WsInfo info;
+  if (!lookup(ws, n_bs, &info)) return DSCALE_ERR_WORKSPACE;
+  cudaError_t e = launch_lm_head(ws, n_bs, hidden, weight, hidden_dim, vocab, accept_len, next_anchor,
+                                 out_tokens, out_len, ctx_len_inout, row_max, info.n_kv_heads,
+                                 info.num_ctas, (cudaStream_t)stream);
+  if (e == cudaErrorNotSupported) return DSCALE_ERR_UNSUPPORTED;
+  return e == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
+}
+
 int dscale_accept_sampling(void* ws, int n_bs, const float* logits, int64_t ld, int vocab,
                            float temperature, const float* u_accept, const float* u_draw,
                            int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
@@ -294,6 +312,7 @@ int dscale_launches_per_call(int which) {
     case 3: return 1;   // attn_simt_kernel
     case 4: return 1;   // attn_padded_kernel
     case 5: return 2;   // sample_stats_kernel + sample_draw_kernel
+    case 6: return 1;   // lm_head_kernel
     default: return 0;
   }
 }

@@ -77,6 +77,12 @@ struct SampleArgs {
 };
 cudaError_t launch_accept_sampling(const SampleArgs& a, cudaStream_t stream);
 
+// fused LM head + argmax + greedy acceptance (tensor cores)
+cudaError_t launch_lm_head(void* ws, int n_bs, const void* hidden, const void* weight, int hidden_dim,
+                           int vocab, int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
+                           int32_t* out_len, int32_t* ctx_len_inout, float* row_max, int n_kv_heads,
+                           int num_ctas, cudaStream_t stream);
+
 // comparison baseline: unpacked W = 16, one 128-row tile per (request, q-head)
 cudaError_t launch_attn_padded(void* ws, int n_bs, const void* q_unpacked, const void* k_cache,
                                const void* v_cache, const int32_t* block_table, int max_pages,

@@ -23,12 +23,12 @@ constexpr int kTcRows = 64;       // rows of the tensor-core query tile (GQA gro
 // header words (int32)
 enum HdrWord {
   H_STATUS = 0, H_N_LIVE = 1, H_M_LIVE = 2, H_TOTAL_TILES = 3, H_ACCEPT_TICKET = 4,
-  H_MAGIC = 5, H_SAMPLE_TICKET = 6, H_WORDS = 64
+  H_MAGIC = 5, H_SAMPLE_TICKET = 6, H_LM_TICKET = 7, H_WORDS = 64
 };
 
 struct WsLayout {
   size_t hdr, k, k0, offset, q_start, q_end, tokens, positions, kv_refs, row_req, top1,
-      kv_len, tile_prefix, qscores, amax_val, amax_idx, smp_m, smp_s, row_m, row_z, row_flag, req_row, req_rej, pair_cnt, pad_cnt,
+      kv_len, tile_prefix, qscores, amax_val, amax_idx, smp_m, smp_s, row_m, row_z, row_flag, req_row, req_rej, pair_cnt, pad_cnt, lm_val, lm_idx,
       part_o, part_ml, trace, total;
 };
 
@@ -66,6 +66,9 @@ __host__ __device__ inline WsLayout ws_layout(int n_bs, int n_kv_heads, int num_
   L.pair_cnt = o;    o = ws_align(o + size_t(n_bs) * n_kv_heads * 4);
   // arrival counters of the padded comparison kernel: one per (request, q-head), group <= 8
   L.pad_cnt = o;     o = ws_align(o + size_t(n_bs) * n_kv_heads * 8 * 4);
+  // fused LM head: one (max logit, index) partial per (packed row, CTA)
+  L.lm_val = o;      o = ws_align(o + m_bs * size_t(num_ctas) * 4);
+  L.lm_idx = o;      o = ws_align(o + m_bs * size_t(num_ctas) * 4);
   // split-KV partials of the attention kernel: per CTA two slots (the segment
   // that starts its range and the one that ends it), each kTcRows rows of
   // (128 fp32 accumulators) plus (row max, row sum)
