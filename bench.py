@@ -46,6 +46,17 @@ def measured_peak():
     return 6650.0, "fallback"
 
 
+def measured_bf16_peak():
+    """Dense bf16 tensor peak in TFLOP/s for a kernel timed alone (burst figure)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["bf16_tflops"])
+        except Exception:
+            pass
+    return 1590.0
+
+
 def recorded_traffic(workload: str):
     """DRAM bytes per attention launch from the committed ncu summary, if any."""
     p = os.path.join(ROOT, "profiles", "attn_tc_traffic.json")
@@ -367,7 +378,10 @@ def run_ours(args, rank, world, local_rank):
             lm_flops = 2.0 * 8 * n * cfg.vocab * args.lm_hidden
             lm = {"us": lm_ms * 1e3, "hidden": args.lm_hidden, "bytes": lm_bytes,
                   "gbs": lm_bytes / (lm_ms * 1e-3) / 1e9, "tflops": lm_flops / (lm_ms * 1e-3) / 1e12,
-                  "library_gemm_logits_only_us": gemm_ms * 1e3}
+                  "library_gemm_logits_only_us": gemm_ms * 1e3,
+                  # both roofs lie close together at 256 rows: report the fraction of each
+                  "frac_of_hbm_peak": lm_bytes / (lm_ms * 1e-3) / 1e9 / measured_peak()[0],
+                  "frac_of_bf16_peak": lm_flops / (lm_ms * 1e-3) / 1e12 / measured_bf16_peak()}
             del w_lm, h_lm, lg
 
         # ---- timed region 3: end to end through the host-buffer C ABI call ----

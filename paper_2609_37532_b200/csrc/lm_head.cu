@@ -5,19 +5,21 @@
 // written and read back, next to 1.24 GB of bf16 weights that have to be read
 // anyway).  A dense contraction: this one belongs on the tensor cores.
 //
-// Each CTA of a persistent grid owns a contiguous range of vocabulary columns,
-// cut into equal tiles of n_tile <= 256 columns (a multiple of 16, chosen on the
-// host so that all CTAs get the same number of equal tiles).  For a tile it
-// accumulates all <= 4 row tiles of 128 packed rows at once in TMEM
-// (m_tiles x n_tile fp32 columns), so every weight element is read from HBM
-// exactly once; the hidden rows (2 MB) are re-read from L2.
-//   warp 4   TMA producer: per 64-wide k step the hidden boxes [128 rows][64]
-//            and the weight box [n_tile rows][64], 128-byte swizzle, ring of
-//            shared-memory stages with mbarrier expect-tx.
+// Up to 128 packed rows: each CTA of a persistent grid owns a contiguous range of
+// vocabulary columns, cut into equal tiles of n_tile <= 256 columns (a multiple
+// of 16, chosen on the host so that all CTAs get the same number of equal tiles),
+// and accumulates a tile in TMEM, so every weight element is read from HBM
+// exactly once; the hidden rows are re-read from L2.
+//   warp 4   TMA producer: per 64-wide k step the hidden box [128 rows][64] and
+//            the weight box [n_tile rows][64], 128-byte swizzle, ring of
+//            shared-memory stages with mbarrier expect-tx; one lane per box.
 //   warp 5   one thread issues tcgen05.mma (M128, N = n_tile, K16 x 4 per step).
 //   warps 0-3  epilogue: thread = packed row; tcgen05.ld 32 columns at a time,
 //            running (max, first index); after the CTA's last tile one partial
 //            per (row, CTA) goes to the workspace.
+// More than 128 rows: pairs of CTAs (cta_group::2, further down), which halve the
+// hidden-state traffic per weight byte.  The one-CTA kernel also exists for 2-4
+// row tiles and serves when no CTA pair can be resident.
 // The last CTA to finish (ticket, nobody waits) merges the partials in vocabulary
 // order -- so equal maxima resolve to the lowest index -- and runs the acceptance
 // loop of the "Prefix verifier" paragraph.
@@ -81,6 +83,118 @@ struct LmArgs {
   float* row_max;          // nullable [8 n_bs]: the winning logit of every live row
 };
 
+// Running (max, first index) over the n fp32 accumulator columns at TMEM address
+// `taddr` of this thread's lane; column x is vocabulary entry col0 + x.  The
+// loads are warp-collective, so dead rows load too and only skip the compare.
+__device__ __forceinline__ void scan_acc(uint32_t taddr, int n, int col0, int vocab, bool live,
+                                         float& best, int& best_i) {
+  for (int ch = 0; ch + 32 <= n; ch += 32) {
+    float v[32];
+    tmem_ld32(taddr + ch, v);
+    if (live) {
+#pragma unroll
+      for (int x = 0; x < 32; ++x) {
+        const int col = col0 + ch + x;
+        if (col < vocab && v[x] > best) { best = v[x]; best_i = col; }
+      }
+    }
+  }
+  if (n & 16) {
+    const int ch = n & ~31;
+    float v[16];
+    tmem_ld16(taddr + ch, v);
+    if (live) {
+#pragma unroll
+      for (int x = 0; x < 16; ++x) {
+        const int col = col0 + ch + x;
+        if (col < vocab && v[x] > best) { best = v[x]; best_i = col; }
+      }
+    }
+  }
+}
+
+// After a CTA's last tile: one (max, index) partial per (row, part) goes to the
+// workspace; the last CTA to finish (ticket, nobody waits) merges the parts in
+// vocabulary order -- so equal maxima resolve to the lowest index -- and runs the
+// acceptance loop of the "Prefix verifier" paragraph.  Called by the 128 epilogue
+// threads of a CTA; `rows[m]` is the packed row this thread holds in best[m].
+__device__ __forceinline__ void lm_finish(const LmArgs& a, const WsLayout& L, int* hdr, int m_live,
+                                          const float* best, const int* best_i, const int* rows, int n_m,
+                                          int part, int n_parts, int n_ctas, bool ok, uint32_t bar_group,
+                                          volatile int* s_abort, int* s_last, int tid) {
+  float* pv = ws_ptr<float>(a.ws, L.lm_val);
+  int* pi = ws_ptr<int>(a.ws, L.lm_idx);
+#pragma unroll
+  for (int m = 0; m < 4; ++m) {
+    if (m < n_m && rows[m] < m_live) {
+      pv[(size_t)rows[m] * n_parts + part] = best[m];
+      pi[(size_t)rows[m] * n_parts + part] = best_i[m];
+    }
+  }
+  __threadfence();
+  unsigned group_phase = 0;
+  auto group_sync = [&]() -> bool {                   // bounded barrier of the 128 epilogue threads
+    mbar_arrive(bar_group);
+    const bool r = mbar_wait(bar_group, group_phase & 1, s_abort);
+    ++group_phase;
+    return r;
+  };
+  ok = ok && group_sync();
+  if (ok && tid == 0) *s_last = (atomicAdd(&hdr[H_LM_TICKET], 1) == n_ctas - 1);
+  ok = ok && group_sync();
+  if (!(ok && *s_last)) return;
+  __threadfence();
+  if (tid == 0) hdr[H_LM_TICKET] = 0;                 // ready for the next launch
+  int* top1 = ws_ptr<int>(a.ws, L.top1);
+  const int m_bs = kHalfW * a.n_bs;
+  for (int r = tid; r < m_bs; r += kEpiThreads) {
+    int bi = 0;
+    if (r < m_live) {
+      float bv = -INFINITY;
+      bi = INT_MAX;
+      for (int cc = 0; cc < n_parts; ++cc) {
+        const float v = __ldcg(&pv[(size_t)r * n_parts + cc]);
+        const int i2 = __ldcg(&pi[(size_t)r * n_parts + cc]);
+        if (v > bv || (v == bv && i2 < bi)) { bv = v; bi = i2; }
+      }
+      if (bi == INT_MAX) bi = 0;
+      if (a.row_max) a.row_max[r] = bv;
+    }
+    top1[r] = bi;
+  }
+  ok = group_sync();
+  const int N = hdr[H_N_LIVE];
+  const int* wk = ws_ptr<int>(a.ws, L.k);
+  const int* woff = ws_ptr<int>(a.ws, L.offset);
+  const int* wtok = ws_ptr<int>(a.ws, L.tokens);
+  if (ok && tid < a.n_bs) {
+    const int i = tid;
+    int32_t* ot = a.out_tokens + i * kW;
+    if (i < N) {
+      const int ki = wk[i], oi = woff[i];
+      int acc = 0;
+      while (acc < ki - 1 && top1[oi + acc] == wtok[oi + acc + 1]) ++acc;
+      const int nxt = top1[oi + acc];
+      for (int j = 0; j < kW; ++j) ot[j] = j < acc ? wtok[oi + 1 + j] : (j == acc ? nxt : -1);
+      a.accept_len[i] = acc;
+      a.next_anchor[i] = nxt;
+      a.out_len[i] = acc + 1;
+      if (a.ctx_len_inout) a.ctx_len_inout[i] += acc + 1;
+    } else {
+      for (int j = 0; j < kW; ++j) ot[j] = -1;
+      a.accept_len[i] = 0;
+      a.next_anchor[i] = -1;
+      a.out_len[i] = 0;
+    }
+  }
+}
+
+// Everything the two single-thread issue loops touch per k step is kept in
+// registers and advanced incrementally (ring slot, phase, descriptor words): a
+// lone thread retires a dependent instruction every few cycles, so an integer
+// division or a descriptor rebuilt from scratch in those loops costs more than
+// the MMAs they issue.
+template <int M_TILES>
 __global__ void __launch_bounds__(kThreads, 1)
 lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtensorMap tm_a,
                const __grid_constant__ CUtensorMap tm_b) {
@@ -92,7 +206,8 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm + off_bar + 256);
   volatile int* s_abort = reinterpret_cast<volatile int*>(sm + off_bar + 260);
   int* s_last = reinterpret_cast<int*>(sm + off_bar + 264);
-  auto bar = [&](int b) { return base + off_bar + 8u * b; };
+  const uint32_t bar0 = base + off_bar;
+  auto bar = [&](int b) { return bar0 + 8u * b; };
   const int B_FULL = 0, B_EMPTY = sh.stages, B_ACC_FULL = 2 * sh.stages, B_ACC_EMPTY = B_ACC_FULL + 1,
             B_GROUP = B_ACC_FULL + 2;
 
@@ -127,26 +242,28 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
   int my_tiles = 0;
   for (int t = 0; t < sh.tiles_per_cta; ++t) my_tiles += (col_begin + t * sh.n_tile < a.vocab);
   const int k_steps = a.hidden_dim / kKStep;
-  const uint32_t a_box_bytes = (uint32_t)sh.a_rows * kKStep * 2;
-  const uint32_t b_box_bytes = (uint32_t)sh.n_tile * kKStep * 2;
 
   if (warp == 4) {
     // ===================================================== TMA producer
-    if (lane == 0) {
-      unsigned u = 0;
-      bool ok = true;
-      for (int t = 0; t < my_tiles && ok; ++t) {
-        const int col0 = col_begin + t * sh.n_tile;
-        for (int kb = 0; kb < k_steps && ok; ++kb, ++u) {
-          const int slot = u % sh.stages;
-          ok = mbar_wait(bar(B_EMPTY + slot), ((u / sh.stages) & 1) ^ 1, s_abort);
-          if (!ok) break;
-          mbar_expect_tx(bar(B_FULL + slot), sh.m_tiles * a_box_bytes + b_box_bytes);
-          const uint32_t st = base + slot * sh.stage_bytes;
-          for (int m = 0; m < sh.m_tiles; ++m)
-            tma_load_2d(st + m * kATile, &tm_a, bar(B_FULL + slot), kb * kKStep, m * 128);
-          tma_load_2d(st + sh.m_tiles * kATile, &tm_b, bar(B_FULL + slot), kb * kKStep, col0);
-        }
+    // lane m < M_TILES copies hidden box m, lane M_TILES the weight box: the
+    // copies of a k step are issued by one warp instruction
+    const bool is_a = lane < M_TILES, is_b = lane == M_TILES;
+    const CUtensorMap* map = is_a ? &tm_a : &tm_b;
+    const uint32_t dst_off = (is_a ? lane : M_TILES) * kATile;
+    const uint32_t tx_bytes = M_TILES * (uint32_t)sh.a_rows * kKStep * 2 + (uint32_t)sh.n_tile * kKStep * 2;
+    int slot = 0;
+    uint32_t empty_parity = 1, st = base;
+    bool ok = true;
+    for (int t = 0; t < my_tiles && ok; ++t) {
+      const int c1 = is_a ? lane * 128 : col_begin + t * sh.n_tile;
+      for (int kb = 0; kb < k_steps; ++kb) {
+        ok = mbar_wait(bar(B_EMPTY + slot), empty_parity, s_abort);
+        if (!ok) break;
+        if (lane == 0) mbar_expect_tx(bar(B_FULL + slot), tx_bytes);
+        __syncwarp();
+        if (is_a || is_b) tma_load_2d(st + dst_off, map, bar(B_FULL + slot), kb * kKStep, c1);
+        st += sh.stage_bytes;
+        if (++slot == sh.stages) { slot = 0; empty_parity ^= 1; st = base; }
       }
     }
     __syncwarp();
@@ -155,28 +272,30 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(sh.n_tile >> 3) << 17) |
                              ((128u >> 4) << 24);
-      unsigned u = 0;
+      const uint64_t desc_hi = smem_desc(0, 16, 1024);          // everything but the start address
+      const uint32_t stage_step = (uint32_t)sh.stage_bytes >> 4;
+      int slot = 0;
+      uint32_t full_parity = 0, st_lo = base >> 4;
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
-        ok = mbar_wait(bar(B_ACC_EMPTY), (t & 1) ^ 1, s_abort);      // accumulators drained
+        ok = mbar_wait(bar(B_ACC_EMPTY), (t & 1) ^ 1, s_abort);        // accumulators drained
         if (!ok) break;
         tc_fence_after();
-        for (int kb = 0; kb < k_steps && ok; ++kb, ++u) {
-          const int slot = u % sh.stages;
-          ok = mbar_wait(bar(B_FULL + slot), (u / sh.stages) & 1, s_abort);
+        for (int kb = 0; kb < k_steps; ++kb) {
+          ok = mbar_wait(bar(B_FULL + slot), full_parity, s_abort);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t st = base + slot * sh.stage_bytes;
-          const uint32_t b_base = st + sh.m_tiles * kATile;
+          const uint32_t b_lo = st_lo + M_TILES * (kATile >> 4);
 #pragma unroll
           for (int ks = 0; ks < kKStep / 16; ++ks) {
-            const uint64_t bd = smem_desc(b_base + ks * 32, 16, 1024);
-            for (int m = 0; m < sh.m_tiles; ++m) {
-              const uint64_t ad = smem_desc(st + m * kATile + ks * 32, 16, 1024);
-              umma(tmem + m * sh.n_tile, ad, bd, idesc, (kb | ks) != 0);
-            }
+#pragma unroll
+            for (int m = 0; m < M_TILES; ++m)
+              umma(tmem + m * sh.n_tile, desc_hi | (uint64_t)(st_lo + m * (kATile >> 4) + ks * 2),
+                   desc_hi | (uint64_t)(b_lo + ks * 2), idesc, (kb | ks) != 0);
           }
           umma_commit(bar(B_EMPTY + slot));
+          st_lo += stage_step;
+          if (++slot == sh.stages) { slot = 0; full_parity ^= 1; st_lo = base >> 4; }
         }
         if (ok) umma_commit(bar(B_ACC_FULL));
       }
@@ -187,8 +306,9 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
     float best[4];
     int best_i[4];
+    int rows[4];
 #pragma unroll
-    for (int m = 0; m < 4; ++m) { best[m] = -INFINITY; best_i[m] = INT_MAX; }
+    for (int m = 0; m < 4; ++m) { best[m] = -INFINITY; best_i[m] = INT_MAX; rows[m] = m * 128 + tid; }
     bool ok = true;
     for (int t = 0; t < my_tiles && ok; ++t) {
       ok = mbar_wait(bar(B_ACC_FULL), t & 1, s_abort);
@@ -196,106 +316,12 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
       tc_fence_after();
       const int col0 = col_begin + t * sh.n_tile;
 #pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        if (m < sh.m_tiles) {
-          const bool live = m * 128 + tid < m_live;           // warp-uniform only per row; loads are collective
-          for (int ch = 0; ch + 32 <= sh.n_tile; ch += 32) {
-            float v[32];
-            tmem_ld32(t_lane + m * sh.n_tile + ch, v);
-            if (live) {
-#pragma unroll
-              for (int x = 0; x < 32; ++x) {
-                const int col = col0 + ch + x;
-                if (col < a.vocab && v[x] > best[m]) { best[m] = v[x]; best_i[m] = col; }
-              }
-            }
-          }
-          if (sh.n_tile & 16) {
-            const int ch = sh.n_tile & ~31;
-            float v[16];
-            tmem_ld16(t_lane + m * sh.n_tile + ch, v);
-            if (live) {
-#pragma unroll
-              for (int x = 0; x < 16; ++x) {
-                const int col = col0 + ch + x;
-                if (col < a.vocab && v[x] > best[m]) { best[m] = v[x]; best_i[m] = col; }
-              }
-            }
-          }
-        }
-      }
+      for (int m = 0; m < M_TILES; ++m)
+        scan_acc(t_lane + m * sh.n_tile, sh.n_tile, col0, a.vocab, rows[m] < m_live, best[m], best_i[m]);
       tc_fence_before();
       mbar_arrive(bar(B_ACC_EMPTY));
     }
-    // one partial per (row, CTA); CTAs without columns write the neutral element
-    float* pv = ws_ptr<float>(a.ws, L.lm_val);
-    int* pi = ws_ptr<int>(a.ws, L.lm_idx);
-#pragma unroll
-    for (int m = 0; m < 4; ++m) {
-      const int row = m * 128 + tid;
-      if (m < sh.m_tiles && row < m_live) {
-        pv[(size_t)row * C + c] = best[m];
-        pi[(size_t)row * C + c] = best_i[m];
-      }
-    }
-    __threadfence();
-    unsigned group_phase = 0;
-    auto group_sync = [&]() -> bool {                 // bounded barrier of the 128 epilogue threads
-      mbar_arrive(bar(B_GROUP));
-      const bool r = mbar_wait(bar(B_GROUP), group_phase & 1, s_abort);
-      ++group_phase;
-      return r;
-    };
-    ok = ok && group_sync();
-    if (ok && tid == 0) *s_last = (atomicAdd(&hdr[H_LM_TICKET], 1) == C - 1);
-    ok = ok && group_sync();
-    if (ok && *s_last) {
-      // ---- last CTA: merge in vocabulary order, then the acceptance loop
-      __threadfence();
-      if (tid == 0) hdr[H_LM_TICKET] = 0;
-      int* top1 = ws_ptr<int>(a.ws, L.top1);
-      const int m_bs = kHalfW * a.n_bs;
-      for (int r = tid; r < m_bs; r += kEpiThreads) {
-        int bi = 0;
-        if (r < m_live) {
-          float bv = -INFINITY;
-          bi = INT_MAX;
-          for (int cc = 0; cc < C; ++cc) {
-            const float v = __ldcg(&pv[(size_t)r * C + cc]);
-            const int i2 = __ldcg(&pi[(size_t)r * C + cc]);
-            if (v > bv || (v == bv && i2 < bi)) { bv = v; bi = i2; }
-          }
-          if (bi == INT_MAX) bi = 0;
-          if (a.row_max) a.row_max[r] = bv;
-        }
-        top1[r] = bi;
-      }
-      ok = group_sync();
-      const int N = hdr[H_N_LIVE];
-      const int* wk = ws_ptr<int>(a.ws, L.k);
-      const int* woff = ws_ptr<int>(a.ws, L.offset);
-      const int* wtok = ws_ptr<int>(a.ws, L.tokens);
-      if (ok && tid < a.n_bs) {
-        const int i = tid;
-        int32_t* ot = a.out_tokens + i * kW;
-        if (i < N) {
-          const int ki = wk[i], oi = woff[i];
-          int acc = 0;
-          while (acc < ki - 1 && top1[oi + acc] == wtok[oi + acc + 1]) ++acc;
-          const int nxt = top1[oi + acc];
-          for (int j = 0; j < kW; ++j) ot[j] = j < acc ? wtok[oi + 1 + j] : (j == acc ? nxt : -1);
-          a.accept_len[i] = acc;
-          a.next_anchor[i] = nxt;
-          a.out_len[i] = acc + 1;
-          if (a.ctx_len_inout) a.ctx_len_inout[i] += acc + 1;
-        } else {
-          for (int j = 0; j < kW; ++j) ot[j] = -1;
-          a.accept_len[i] = 0;
-          a.next_anchor[i] = -1;
-          a.out_len[i] = 0;
-        }
-      }
-    }
+    lm_finish(a, L, hdr, m_live, best, best_i, rows, M_TILES, c, C, C, ok, bar(B_GROUP), s_abort, s_last, tid);
   }
 
   tc_fence_before();
@@ -304,6 +330,237 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
   if (warp == 5) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------
+// CTA-pair variant for more than 128 packed rows (cta_group::2).
+//
+// With one CTA per tile the 256 x 4096 hidden block is re-read from L2 for every
+// 208 vocabulary columns and takes more than half of the shared-memory ring, so
+// the weight bytes in flight per SM -- what bounds a stream at HBM latency --
+// are few.  A pair of CTAs on neighbouring SMs issues M = 256 MMAs instead: each
+// CTA stages only ITS 128 hidden rows and HALF of every weight tile, the tensor
+// cores read the other half from the partner's shared memory, and each CTA
+// accumulates its 128 rows x N columns in its own TMEM.  Per pass a pair covers
+// 256 rows x 2N columns (rows <= 256) or 512 rows x N columns.
+//   both CTAs   warp 4: TMA producer into the own ring; the transaction bytes of
+//               both CTAs complete on the LEADER's full barrier.
+//               warps 0-3: epilogue over the own 128 rows per row block.
+//   leader      warp 5: issues the MMAs; tcgen05.commit arrives on the empty /
+//               accumulator-full barriers of both CTAs.
+// Every wait is bounded; the two CTAs meet at a cluster barrier before the
+// tensor memory is released.
+struct PairShape {
+  int m_pairs;        // row blocks of 256 packed rows (1 or 2)
+  int n_acc;          // accumulators per row block (2 or 1): m_pairs * n_acc = 2
+  int n;              // N of one MMA (multiple of 16, <= 256); each CTA stages n / 2 weight rows
+  int passes;
+  int cols_per_pair;  // n * n_acc * passes
+  int stages;
+  int stage_bytes;
+  int b_bytes;        // one staged half weight tile
+  int smem_bytes;
+};
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into the own shared memory whose bytes complete on a barrier that may
+// live in the partner CTA (cluster address)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster,
+                                                 int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void umma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(bar_cluster) : "memory");
+}
+
+template <int M_PAIRS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+lm_head_pair_kernel(LmArgs a, WsLayout L, PairShape sh, const __grid_constant__ CUtensorMap tm_a,
+                    const __grid_constant__ CUtensorMap tm_b) {
+  constexpr int N_ACC = 2 / M_PAIRS;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t raw = smem_u32(smem_dyn);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* sm = smem_dyn + (base - raw);
+  const int off_bar = sh.stages * sh.stage_bytes;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm + off_bar + 256);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(sm + off_bar + 260);
+  int* s_last = reinterpret_cast<int*>(sm + off_bar + 264);
+  const uint32_t bar0 = base + off_bar;
+  auto bar = [&](int b) { return bar0 + 8u * b; };
+  const int B_FULL = 0, B_EMPTY = sh.stages, B_ACC_FULL = 2 * sh.stages, B_ACC_EMPTY = B_ACC_FULL + 1,
+            B_GROUP = B_ACC_FULL + 2;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_rank();              // 0 = leader (issues the MMAs)
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  int* hdr = ws_ptr<int>(a.ws, L.hdr);
+  const int m_live = hdr[H_M_LIVE];
+
+  if (tid == 0) {
+    for (int s = 0; s < sh.stages; ++s) { mbar_init(bar(B_FULL + s), 1); mbar_init(bar(B_EMPTY + s), 1); }
+    mbar_init(bar(B_ACC_FULL), 1);
+    mbar_init(bar(B_ACC_EMPTY), 2 * kEpiThreads);    // the epilogue threads of both CTAs
+    mbar_init(bar(B_GROUP), kEpiThreads);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;"
+                 ::"r"(smem_u32(s_tmem)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  if (warp == 4 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b) : "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                 // the partner's barriers exist before anything signals them
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+
+  const int col_begin = pair * sh.cols_per_pair;
+  const int pass_cols = sh.n * N_ACC;
+  int my_passes = 0;
+  for (int t = 0; t < sh.passes; ++t) my_passes += (col_begin + t * pass_cols < a.vocab);
+  const int k_steps = a.hidden_dim / kKStep;
+  const int half = sh.n >> 1;
+
+  if (warp == 4) {
+    // ===================================================== TMA producer (both CTAs)
+    // lane p < M_PAIRS copies this CTA's 128 hidden rows of row block p, lane
+    // M_PAIRS + j its half of the weight tile of accumulator j
+    const bool is_a = lane < M_PAIRS, is_b = lane >= M_PAIRS && lane < M_PAIRS + N_ACC;
+    const int j = lane - M_PAIRS;
+    const CUtensorMap* map = is_a ? &tm_a : &tm_b;
+    const uint32_t dst_off = is_a ? lane * kATile : M_PAIRS * kATile + j * sh.b_bytes;
+    const uint32_t payload = (uint32_t)M_PAIRS * kATile + (uint32_t)N_ACC * half * kKStep * 2;
+    const uint32_t full0 = map_to_cta(bar(B_FULL), 0);           // the leader's full barriers
+    int slot = 0;
+    uint32_t empty_parity = 1, st = base;
+    bool ok = true;
+    for (int t = 0; t < my_passes && ok; ++t) {
+      const int c1 = is_a ? lane * 256 + (int)rank * 128 : col_begin + t * pass_cols + j * sh.n + (int)rank * half;
+      for (int kb = 0; kb < k_steps; ++kb) {
+        ok = mbar_wait(bar(B_EMPTY + slot), empty_parity, s_abort);
+        if (!ok) break;
+        if (lane == 0 && rank == 0) mbar_expect_tx(bar(B_FULL + slot), 2 * payload);
+        __syncwarp();
+        if (is_a || is_b) tma_load_2d_pair(st + dst_off, map, full0 + 8u * slot, kb * kKStep, c1);
+        st += sh.stage_bytes;
+        if (++slot == sh.stages) { slot = 0; empty_parity ^= 1; st = base; }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    // ===================================================== MMA issuer (leader only)
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(sh.n >> 3) << 17) |
+                             ((256u >> 4) << 24);
+      const uint64_t desc_hi = smem_desc(0, 16, 1024);
+      const uint32_t stage_step = (uint32_t)sh.stage_bytes >> 4, b_step = (uint32_t)sh.b_bytes >> 4;
+      const uint32_t peer_bar0 = map_to_cta(bar0, 1);
+      int slot = 0;
+      uint32_t full_parity = 0, st_lo = base >> 4;
+      bool ok = true;
+      for (int t = 0; t < my_passes && ok; ++t) {
+        ok = mbar_wait(bar(B_ACC_EMPTY), (t & 1) ^ 1, s_abort);        // both CTAs drained their accumulators
+        if (!ok) break;
+        tc_fence_after();
+        for (int kb = 0; kb < k_steps; ++kb) {
+          ok = mbar_wait(bar(B_FULL + slot), full_parity, s_abort);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t b_lo = st_lo + M_PAIRS * (kATile >> 4);
+#pragma unroll
+          for (int ks = 0; ks < kKStep / 16; ++ks) {
+#pragma unroll
+            for (int p = 0; p < M_PAIRS; ++p) {
+#pragma unroll
+              for (int j = 0; j < N_ACC; ++j)
+                umma_pair(tmem + (p * N_ACC + j) * sh.n, desc_hi | (uint64_t)(st_lo + p * (kATile >> 4) + ks * 2),
+                          desc_hi | (uint64_t)(b_lo + j * b_step + ks * 2), idesc, (kb | ks) != 0);
+            }
+          }
+          umma_commit_pair(bar(B_EMPTY + slot));
+          umma_commit_pair(peer_bar0 + 8u * (B_EMPTY + slot));
+          st_lo += stage_step;
+          if (++slot == sh.stages) { slot = 0; full_parity ^= 1; st_lo = base >> 4; }
+        }
+        if (ok) {
+          umma_commit_pair(bar(B_ACC_FULL));
+          umma_commit_pair(peer_bar0 + 8u * B_ACC_FULL);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ===================================================== epilogue warps 0-3 (both CTAs)
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t acc_empty = map_to_cta(bar(B_ACC_EMPTY), 0);
+    float best[4];
+    int best_i[4];
+    int rows[4];
+#pragma unroll
+    for (int m = 0; m < 4; ++m) { best[m] = -INFINITY; best_i[m] = INT_MAX; rows[m] = m * 256 + (int)rank * 128 + tid; }
+    bool ok = true;
+    for (int t = 0; t < my_passes && ok; ++t) {
+      ok = mbar_wait(bar(B_ACC_FULL), t & 1, s_abort);
+      if (!ok) break;
+      tc_fence_after();
+      const int col0 = col_begin + t * pass_cols;
+#pragma unroll
+      for (int p = 0; p < M_PAIRS; ++p) {
+#pragma unroll
+        for (int j = 0; j < N_ACC; ++j)
+          scan_acc(t_lane + (p * N_ACC + j) * sh.n, sh.n, col0 + j * sh.n, a.vocab, rows[p] < m_live, best[p],
+                   best_i[p]);
+      }
+      tc_fence_before();
+      mbar_arrive_cluster(acc_empty);
+    }
+    lm_finish(a, L, hdr, m_live, best, best_i, rows, M_PAIRS, pair, n_pairs, (int)gridDim.x, ok,
+              bar(B_GROUP), s_abort, s_last, tid);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && *s_abort) atomicOr(&hdr[H_STATUS], 8 /*TIMEOUT*/);
+  cluster_sync_all();                                 // nobody leaves while the partner may still touch this CTA
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
   }
 }
 
@@ -358,10 +615,58 @@ LmShape plan(int n_bs, int vocab, int num_ctas) {
   return s;
 }
 
+PairShape plan_pair(int n_bs, int vocab, int pairs) {
+  PairShape s;
+  const int rows = kHalfW * n_bs;
+  s.m_pairs = (rows + 255) / 256;
+  s.n_acc = 2 / s.m_pairs;
+  int cols = (vocab + pairs - 1) / pairs;
+  const int per_pass_max = 256 * s.n_acc;
+  s.passes = (cols + per_pass_max - 1) / per_pass_max;
+  const int per_acc = (cols + s.passes * s.n_acc - 1) / (s.passes * s.n_acc);
+  s.n = (per_acc + 15) & ~15;
+  if (s.n < 32) s.n = 32;
+  s.cols_per_pair = s.n * s.n_acc * s.passes;
+  s.b_bytes = (s.n / 2) * kKStep * 2;                 // n / 2 rows of 128 bytes: a multiple of 1024
+  s.stage_bytes = s.m_pairs * kATile + s.n_acc * s.b_bytes;
+  s.stages = (222 * 1024) / s.stage_bytes;
+  if (s.stages > 4) s.stages = 4;                     // measured: a fifth stage does not pay
+  s.smem_bytes = s.stages * s.stage_bytes + 512 + 1024;
+  return s;
+}
+
+// CTA pairs that can be resident at once with the ring at its largest (one CTA
+// per SM either way); a grid beyond it would run a second, nearly empty wave.
+int resident_pairs(int num_ctas) {
+  static int cached = -1;
+  if (cached < 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((num_ctas / 2) * 2);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = 224 * 1024;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, lm_head_pair_kernel<1>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    cached = n;
+  }
+  const int want = num_ctas / 2;
+  return cached < want ? cached : want;
+}
+
 }  // namespace
 
 cudaError_t lm_head_prepare() {
-  return cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  const void* fns[] = {(const void*)lm_head_kernel<1>, (const void*)lm_head_kernel<2>,
+                       (const void*)lm_head_kernel<3>, (const void*)lm_head_kernel<4>,
+                       (const void*)lm_head_pair_kernel<1>, (const void*)lm_head_pair_kernel<2>};
+  for (const void* f : fns) {
+    cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 cudaError_t launch_lm_head(void* ws, int n_bs, const void* hidden, const void* weight, int hidden_dim,
@@ -369,15 +674,33 @@ cudaError_t launch_lm_head(void* ws, int n_bs, const void* hidden, const void* w
                            int32_t* out_len, int32_t* ctx_len_inout, float* row_max, int n_kv_heads,
                            int num_ctas, cudaStream_t stream) {
   WsLayout L = ws_layout(n_bs, n_kv_heads, num_ctas);
+  LmArgs a{ws, n_bs, hidden_dim, vocab, accept_len, next_anchor, out_tokens, out_len, ctx_len_inout, row_max};
+  CUtensorMap ta, tb;
+  const int pairs = kHalfW * n_bs > 128 ? resident_pairs(num_ctas) : 0;
+  if (pairs >= 1) {
+    // more than one row tile: CTA pairs
+    PairShape ps = plan_pair(n_bs, vocab, pairs);
+    if (ps.stages < 2) return cudaErrorNotSupported;
+    const int b_box = ps.n / 2 < vocab ? ps.n / 2 : vocab;
+    if (!encode_2d(&ta, hidden, hidden_dim, kHalfW * n_bs, 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B) ||
+        !encode_2d(&tb, weight, hidden_dim, vocab, b_box, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+      return cudaErrorNotSupported;
+    if (ps.m_pairs == 1) lm_head_pair_kernel<1><<<pairs * 2, kThreads, ps.smem_bytes, stream>>>(a, L, ps, ta, tb);
+    else lm_head_pair_kernel<2><<<pairs * 2, kThreads, ps.smem_bytes, stream>>>(a, L, ps, ta, tb);
+    return cudaGetLastError();
+  }
   LmShape sh = plan(n_bs, vocab, num_ctas);
   if (sh.stages < 2 || sh.n_tile < 16) return cudaErrorNotSupported;
-  CUtensorMap ta, tb;
   if (!encode_2d(&ta, hidden, hidden_dim, kHalfW * n_bs, sh.a_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B) ||
       !encode_2d(&tb, weight, hidden_dim, vocab, sh.n_tile < vocab ? sh.n_tile : vocab,
-                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B))
+                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
     return cudaErrorNotSupported;
-  LmArgs a{ws, n_bs, hidden_dim, vocab, accept_len, next_anchor, out_tokens, out_len, ctx_len_inout, row_max};
-  lm_head_kernel<<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb);
+  switch (sh.m_tiles) {
+    case 1: lm_head_kernel<1><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb); break;
+    case 2: lm_head_kernel<2><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb); break;
+    case 3: lm_head_kernel<3><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb); break;
+    default: lm_head_kernel<4><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb); break;
+  }
   return cudaGetLastError();
 }
 
