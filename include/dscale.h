@@ -235,7 +235,8 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
 /*
  * Fused LM head + greedy prefix verification: dscale_accept without the logits.
  * The target token of packed row s is argmax_v sum_h hidden[s][h] * weight[v][h]
- * (the LM head applied to the M = 8N packed rows DVL leaves, Section 3.3), computed
+ * (the LM head applied to the M = 8N packed rows DVL leaves: Section 2.2 and the
+ * last sentence of Section 3.2), computed
  * on the tensor cores tile by tile with a running (max, first index) per row, so
  * the 8N x V logits are never written; then the same acceptance loop and outputs
  * as dscale_accept (Algorithm 2, lines 21-26).
@@ -245,6 +246,13 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
  *   row_max  nullable fp32 [8 n_bs]: receives the winning logit of every live row
  * Products are accumulated in fp32; two logits closer than fp32 rounding of the
  * dot product may resolve differently from an exact evaluation.
+ * All pointers are device pointers owned by the caller; hidden and weight must be
+ * 16-byte aligned.  dscale_alloc_verify must have run on ws for this step.  Outputs
+ * as for dscale_accept.  One launch on `stream`, no allocation, no synchronisation;
+ * the first call on a device queries the occupancy of the CTA-pair kernel and
+ * should come before any stream capture.  Returns DSCALE_ERR_UNSUPPORTED for
+ * hidden_dim % 64 != 0 or vocab < 16, DSCALE_ERR_WORKSPACE for an unknown ws,
+ * DSCALE_ERR_INVALID_ARG for null or misaligned pointers.
  */
 int dscale_lm_head_accept(void* ws, int n_bs, const void* hidden, const void* weight, int hidden_dim,
                           int vocab, int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
