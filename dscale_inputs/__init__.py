@@ -223,6 +223,38 @@ def make_lm_head_unpacked(req: dict, hidden_dim: int, device: str = "cpu"):
     return weight, hidden.to(torch.bfloat16)
 
 
+def make_predictor_inputs(req: dict, hidden_dim: int, device: str = "cpu") -> dict:
+    """Inputs of the acceptance-predictor front end, shape-faithful with seeded
+    random parameters (the trained predictor and the fixed projections are not
+    published).  Drafter logits fp32 [n_bs, 15, ld] (ld = vocab rounded up to a
+    multiple of 4, padding NaN): N(-3, 2^2) with the drafted token of each
+    position lifted by 6, so it is the drafter's top-1 as in the paper's
+    deterministic drafter; drafter hidden states bf16 [n_bs, 15, hidden_dim]
+    N(0,1); fixed projections bf16, N(0, 1/hidden_dim) and N(0, 1/vocab) with a
+    common offset of 0.5/vocab (so the centring term matters); perceptron
+    weights fp32 with fan-in scaling, biases N(0, 0.25)."""
+    cfg = req["cfg"]
+    g = torch.Generator(device=device)
+    g.manual_seed(cfg.seed * 1_000_003 + 15485863)
+    n_bs, V = req["n_bs"], cfg.vocab
+    ld = (V + 3) // 4 * 4
+    kw = dict(generator=g, dtype=torch.float32, device=device)
+    logits = torch.full((n_bs, W - 1, ld), float("nan"), dtype=torch.float32, device=device)
+    logits[:, :, :V] = torch.randn((n_bs, W - 1, V), **kw) * 2.0 - 3.0
+    draft = torch.as_tensor(req["draft_tokens"]).to(device).long()
+    idx = draft[:, 1:].unsqueeze(-1)                                   # candidate of slot p + 1
+    logits.scatter_add_(2, idx, torch.full(idx.shape, 6.0, dtype=torch.float32, device=device))
+    hidden = torch.randn((n_bs, W - 1, hidden_dim), **kw).to(torch.bfloat16)
+    p_hidden = (torch.randn((64, hidden_dim), **kw) / hidden_dim ** 0.5).to(torch.bfloat16)
+    p_logit = (torch.randn((32, V), **kw) / V ** 0.5 + 0.5 / V).to(torch.bfloat16)
+    w1 = torch.randn((64, 1735), **kw) / 1735 ** 0.5
+    b1 = torch.randn((64,), **kw) * 0.5
+    w2 = torch.randn((15, 64), **kw) / 8.0
+    b2 = torch.randn((15,), **kw) * 0.5
+    return dict(draft_logits=logits, draft_hidden=hidden, p_hidden=p_hidden, p_logit=p_logit,
+                w1=w1, b1=b1, w2=w2, b2=b2, ld=ld)
+
+
 def rows_to_packed(unpacked: torch.Tensor, k, offset, n_live: int, m_bs: int,
                    fill: float = 0.0) -> torch.Tensor:
     """Lay the first k_i slot rows of each request at rows offset_i .. of a

@@ -259,6 +259,38 @@ int dscale_lm_head_accept(void* ws, int n_bs, const void* hidden, const void* we
                           int32_t* out_len, int32_t* ctx_len_inout, float* row_max, void* stream);
 
 /*
+ * Acceptance-predictor front end ("Acceptance predictor" paragraph, Eq. 4 and
+ * Eq. 5): the step before dscale_alloc_verify.  For every live request and each
+ * of its 15 new draft positions p:
+ *   confidence (18): top drafter logit; its gaps to the logits of ranks 2..16;
+ *                    log-probability of the top token; entropy of softmax(z)
+ *   hidden projection (64):  p_hidden  . draft_hidden[i][p]
+ *   logit projection (32):   p_logit . (z - mean(z)),  z = draft_logits[i][p]
+ * features_i = [confidence (270, position-major) | hidden projections (960) |
+ * logit projections (480) | batch context (25: entry 0 = N, entry 3 = 1)]: 1735
+ * values; pred_logits[i] = w2 relu(w1 features_i + b1) + b2.  The result is what
+ * dscale_alloc_verify takes as `scores` with scores_are_logits = 1.
+ *
+ *   n_live        device int32[1]
+ *   draft_logits  fp32 [n_bs][15][ld], ld >= vocab, ld % 4 == 0, finite values
+ *   draft_hidden  bf16 [n_bs][15][hidden_dim], hidden_dim % 8 == 0
+ *   p_hidden      bf16 [64][hidden_dim]      p_logit  bf16 [32][vocab]
+ *   w1 fp32 [64][1735], b1 fp32 [64], w2 fp32 [15][64], b2 fp32 [15]
+ *   pred_logits   fp32 [n_bs][15] out; rows of requests >= N are set to 0
+ *   features_out  nullable fp32 [n_bs][1735] out (rows >= N set to 0)
+ * fp32 arithmetic; the logit projection rounds (z - z[0]) to tf32 for the tensor
+ * cores (the centring is applied afterwards, exactly).  All pointers are device
+ * pointers owned by the caller, 16-byte aligned.  Three launches on `stream`, no
+ * allocation, no synchronisation; scratch lives in ws.  vocab >= 16.
+ * Errors: DSCALE_ERR_INVALID_ARG (null / misaligned), DSCALE_ERR_UNSUPPORTED
+ * (shape rules above), DSCALE_ERR_WORKSPACE (unknown ws).
+ */
+int dscale_predict_scores(void* ws, int n_bs, const int32_t* n_live, const float* draft_logits, int64_t ld,
+                          int vocab, const void* draft_hidden, int hidden_dim, const void* p_hidden,
+                          const void* p_logit, const float* w1, const float* b1, const float* w2,
+                          const float* b2, float* pred_logits, float* features_out, void* stream);
+
+/*
  * Prefix verification under a sampling target policy ("Prefix verifier"
  * paragraph, temperature > 0).  P = softmax(logits / temperature) at each packed
  * row.  The candidate x in slot j + 1 is accepted iff u_accept[offset_i + j] < P(x);
@@ -330,7 +362,7 @@ const int32_t* dscale_ws_field(const void* ws, int n_bs, int field);
 
 /* Number of kernels the three stage calls enqueue (for launch accounting):
  * which = 0 alloc, 1 attention, 2 accept, 3 attention (simt), 4 attention (padded),
- * 5 accept (sampling), 6 fused LM head + accept. */
+ * 5 accept (sampling), 6 fused LM head + accept, 7 predictor front end. */
 int dscale_launches_per_call(int which);
 
 #ifdef __cplusplus

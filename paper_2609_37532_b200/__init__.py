@@ -10,8 +10,8 @@ from .build import build as _build
 _build()          # no-op when libdscale.so is newer than its sources; raises if nvcc fails
 
 from .binding import (  # noqa: E402
-    DScaleError, HostStep, VerifyGraphPool, VerifyWorkspace, accept, accept_sampling, accept_static, alloc_verify, lib, lm_head_accept, verify_attn,
+    DScaleError, HostStep, VerifyGraphPool, VerifyWorkspace, accept, accept_sampling, accept_static, alloc_verify, lib, lm_head_accept, predict_scores, verify_attn,
                       verify_attn_padded, verify_attn_simt, WS_FIELDS)
 
-__all__ = ["DScaleError", "HostStep", "VerifyGraphPool", "VerifyWorkspace", "accept", "accept_sampling", "accept_static", "alloc_verify", "lib", "lm_head_accept", "verify_attn",
+__all__ = ["DScaleError", "HostStep", "VerifyGraphPool", "VerifyWorkspace", "accept", "accept_sampling", "accept_static", "alloc_verify", "lib", "lm_head_accept", "predict_scores", "verify_attn",
            "verify_attn_padded", "verify_attn_simt", "WS_FIELDS"]

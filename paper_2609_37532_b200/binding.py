@@ -46,6 +46,8 @@ lib.dscale_verify_attn_padded.restype = _i
 lib.dscale_verify_attn_padded.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i, _i, _vp, _i, _i, _f, _vp, _vp]
 lib.dscale_accept_static.restype = _i
 lib.dscale_accept_static.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _i64, _i, _vp, _vp, _vp, _vp, _vp]
+lib.dscale_predict_scores.restype = _i
+lib.dscale_predict_scores.argtypes = [_vp, _i, _vp, _vp, C.c_int64, _i, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.dscale_lm_head_accept.restype = _i
 lib.dscale_lm_head_accept.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.dscale_accept_sampling.restype = _i
@@ -338,3 +340,20 @@ def lm_head_accept(ws, hidden, weight, accept_len, next_anchor, out_tokens, out_
                                      weight.shape[0], _ptr(accept_len), _ptr(next_anchor), _ptr(out_tokens),
                                      _ptr(out_len), _ptr(ctx_len_inout), _ptr(row_max), _stream()),
            "dscale_lm_head_accept")
+
+
+def predict_scores(ws, n_live, draft_logits, vocab, draft_hidden, p_hidden, p_logit, w1, b1, w2, b2,
+                   pred_logits, features_out=None):
+    """Predictor front end (dscale_predict_scores): drafter logits / hidden states -> predLogits."""
+    _need(n_live, torch.int32, "n_live"); _need(draft_logits, torch.float32, "draft_logits")
+    _need(draft_hidden, torch.bfloat16, "draft_hidden"); _need(p_hidden, torch.bfloat16, "p_hidden")
+    _need(p_logit, torch.bfloat16, "p_logit"); _need(pred_logits, torch.float32, "pred_logits")
+    for n, t in (("w1", w1), ("b1", b1), ("w2", w2), ("b2", b2)):
+        _need(t, torch.float32, n)
+    assert draft_logits.shape[:2] == (ws.n_bs, 15) and draft_hidden.shape[:2] == (ws.n_bs, 15)
+    assert w1.shape == (64, 1735) and w2.shape == (15, 64) and pred_logits.shape == (ws.n_bs, 15)
+    _check(lib.dscale_predict_scores(C.c_void_p(ws.ptr), ws.n_bs, _ptr(n_live), _ptr(draft_logits),
+                                     draft_logits.shape[2], vocab, _ptr(draft_hidden), draft_hidden.shape[2],
+                                     _ptr(p_hidden), _ptr(p_logit), _ptr(w1), _ptr(b1), _ptr(w2), _ptr(b2),
+                                     _ptr(pred_logits), _ptr(features_out), _stream()),
+           "dscale_predict_scores")

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdscale.so")
-SOURCES = ["api.cu", "alloc.cu", "accept.cu", "accept_static.cu", "accept_sampling.cu", "attn_simt.cu", "attn_tc.cu", "attn_padded.cu", "lm_head.cu"]
+SOURCES = ["api.cu", "alloc.cu", "accept.cu", "accept_static.cu", "accept_sampling.cu", "attn_simt.cu", "attn_tc.cu", "attn_padded.cu", "lm_head.cu", "predictor.cu"]
 FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
          "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
 

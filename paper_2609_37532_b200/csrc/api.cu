@@ -68,6 +68,7 @@ int dscale_workspace_init(void* ws, size_t bytes, int n_bs, int n_q_heads, int n
   if (attn_tc_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
   if (attn_padded_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
   if (lm_head_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
+  if (predictor_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
   std::lock_guard<std::mutex> lk(g_mu);
   g_ws[ws] = WsInfo{bytes, n_bs, n_q_heads, n_kv_heads, num_sms};
   return DSCALE_OK;
@@ -257,6 +258,24 @@ int dscale_lm_head_accept(void* ws, int n_bs, const void* hidden, const void* we
   return e == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
 }
 
+int dscale_predict_scores(void* ws, int n_bs, const int32_t* n_live, const float* draft_logits, int64_t ld,
+                          int vocab, const void* draft_hidden, int hidden_dim, const void* p_hidden,
+                          const void* p_logit, const float* w1, const float* b1, const float* w2,
+                          const float* b2, float* pred_logits, float* features_out, void* stream) {
+  if (!ws || !n_live || !draft_logits || !draft_hidden || !p_hidden || !p_logit || !w1 || !b1 || !w2 || !b2 ||
+      !pred_logits)
+    return DSCALE_ERR_INVALID_ARG;
+  if (!aligned(draft_logits, 16) || !aligned(draft_hidden, 16) || !aligned(p_hidden, 16) || !aligned(p_logit, 16))
+    return DSCALE_ERR_INVALID_ARG;
+  if (vocab < 16 || ld < vocab || ld % 4 != 0 || hidden_dim < 8 || hidden_dim % 8 != 0)
+    return DSCALE_ERR_UNSUPPORTED;
+  WsInfo info;
+  if (!lookup(ws, n_bs, &info)) return DSCALE_ERR_WORKSPACE;
+  PredictArgs p{ws, n_bs, n_live, draft_logits, ld, vocab, draft_hidden, hidden_dim, p_hidden, p_logit,
+                w1, b1, w2, b2, pred_logits, features_out, info.n_kv_heads, info.num_ctas};
+  return launch_predictor(p, (cudaStream_t)stream) == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
+}
+
 int dscale_accept_sampling(void* ws, int n_bs, const float* logits, int64_t ld, int vocab,
                            float temperature, const float* u_accept, const float* u_draw,
                            int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
@@ -313,6 +332,7 @@ int dscale_launches_per_call(int which) {
     case 4: return 1;   // attn_padded_kernel
     case 5: return 2;   // sample_stats_kernel + sample_draw_kernel
     case 6: return 1;   // lm_head_kernel
+    case 7: return 3;   // pred_stream_kernel + pred_features_kernel + pred_mlp_kernel
     default: return 0;
   }
 }

@@ -83,6 +83,30 @@ cudaError_t launch_lm_head(void* ws, int n_bs, const void* hidden, const void* w
                            int32_t* out_len, int32_t* ctx_len_inout, float* row_max, int n_kv_heads,
                            int num_ctas, cudaStream_t stream);
 
+// acceptance-predictor front end: drafter logits / hidden states -> predLogits
+struct PredictArgs {
+  void* ws;
+  int n_bs;
+  const int32_t* n_live;
+  const float* draft_logits;   // [n_bs][15][ld]
+  int64_t ld;
+  int vocab;
+  const void* draft_hidden;    // bf16 [n_bs][15][hidden_dim]
+  int hidden_dim;
+  const void* p_hidden;        // bf16 [64][hidden_dim]
+  const void* p_logit;         // bf16 [32][vocab]
+  const float* w1;             // [64][1735]
+  const float* b1;             // [64]
+  const float* w2;             // [15][64]
+  const float* b2;             // [15]
+  float* pred_logits;          // [n_bs][15]
+  float* features_out;         // nullable [n_bs][1735]
+  int n_kv_heads;
+  int num_ctas;
+};
+cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream);
+cudaError_t predictor_prepare();
+
 // comparison baseline: unpacked W = 16, one 128-row tile per (request, q-head)
 cudaError_t launch_attn_padded(void* ws, int n_bs, const void* q_unpacked, const void* k_cache,
                                const void* v_cache, const int32_t* block_table, int max_pages,

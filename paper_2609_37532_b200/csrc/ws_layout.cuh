@@ -19,6 +19,16 @@ constexpr int kMaxNbs = 64;
 constexpr int kTileTok = 128;     // keys per attention tile (8 pages)
 constexpr int kAccMaxChunks = 16; // vocab chunks per row in the argmax
 constexpr int kTcRows = 64;       // rows of the tensor-core query tile (GQA group 4 x 16 slots)
+// acceptance-predictor front end ("Acceptance predictor" paragraph)
+constexpr int kPredPos = 15;          // new draft positions per request
+constexpr int kPredConf = 18;         // confidence values per position
+constexpr int kPredHid = 64;          // hidden-state projection width
+constexpr int kPredLog = 32;          // logit projection width
+constexpr int kPredCtx = 25;          // batch-context values
+constexpr int kPredFeatures = kPredPos * (kPredConf + kPredHid + kPredLog) + kPredCtx;   // 1735
+constexpr int kPredMlp = 64;          // hidden units of the predictor
+constexpr int kPredMaxChunks = 32;    // vocabulary chunks per drafter-logit row
+constexpr int kPredRec = 52;          // 16 top values, (max, sum, sum e z, sum z), 32 projections
 
 // header words (int32)
 enum HdrWord {
@@ -29,7 +39,7 @@ enum HdrWord {
 struct WsLayout {
   size_t hdr, k, k0, offset, q_start, q_end, tokens, positions, kv_refs, row_req, top1,
       kv_len, tile_prefix, qscores, amax_val, amax_idx, smp_m, smp_s, row_m, row_z, row_flag, req_row, req_rej, pair_cnt, pad_cnt, lm_val, lm_idx,
-      part_o, part_ml, trace, total;
+      part_o, part_ml, pred_part, pred_rowsum, pred_feat, trace, total;
 };
 
 __host__ __device__ inline size_t ws_align(size_t x) { return (x + 255) & ~size_t(255); }
@@ -74,6 +84,11 @@ __host__ __device__ inline WsLayout ws_layout(int n_bs, int n_kv_heads, int num_
   // (128 fp32 accumulators) plus (row max, row sum)
   L.part_o = o;      o = ws_align(o + size_t(num_ctas) * 2 * kTcRows * kD * 4);
   L.part_ml = o;     o = ws_align(o + size_t(num_ctas) * 2 * kTcRows * 2 * 4);
+  // predictor front end: per (drafter-logit row, vocabulary chunk) a record of kPredRec
+  // floats, per chunk the row sums of the fixed logit projection, per request the features
+  L.pred_part = o;   o = ws_align(o + size_t(kPredPos) * n_bs * kPredMaxChunks * kPredRec * 4);
+  L.pred_rowsum = o; o = ws_align(o + size_t(kPredMaxChunks) * 32 * 4);
+  L.pred_feat = o;   o = ws_align(o + size_t(n_bs) * kPredFeatures * 4);
   // per-CTA timestamps, written only by builds with -DDSCALE_TRACE
   L.trace = o;       o = ws_align(o + size_t(num_ctas) * 64 * 8);
   L.total = o;

@@ -1,0 +1,120 @@
+"""dscale_predict_scores against the binary64 predictor oracle, feature block by feature block,
+then the predLogits, then the allocation they produce.
+
+Tolerances (fp32 arithmetic on the device, binary64 in the oracle):
+  top logit            exact (a selection)
+  gaps                 1e-6 relative + 1e-6 (one fp32 subtraction)
+  log-prob, entropy    2e-4 (fp32 sums of V fast exponentials)
+  hidden projection    1e-4 + 1e-4 |ref| (bf16 products are exact in fp32; H-term fp32 sum)
+  logit projection     4e-3 + 2e-3 |ref| ((z - z[0]) rounded to tf32: 2^-12 |z'| per element,
+                       random signs, weights of variance 1/V: sigma ~ 4e-4 at |z'| ~ 3)
+  predLogits           3e-3 + 3e-3 |ref| (the above through w1 ~ N(0, 1/1735), w2 ~ N(0, 1/64))
+The allocation is compared bit-exactly with the oracle run on the device's own predLogits."""
+import numpy as np
+import pytest
+import torch
+
+from dscale_inputs import CONFIGS, make_predictor_inputs, make_requests, small_variant
+from gpu_case import ALLOC_FIELDS, StagedRequests, assert_alloc_equal
+from oracle import dvl_alloc as OA
+from oracle import predictor as OP
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(P, cfg, n_bs, hidden_dim, gen_device="cpu"):
+    req = make_requests(cfg, n_bs=n_bs)
+    n, V = req["n_live"], cfg.vocab
+    d = make_predictor_inputs(req, hidden_dim, device=gen_device)
+    host = {k: (v.float().cpu().numpy() if torch.is_tensor(v) else v) for k, v in d.items()}
+    exp = OP.predict(host["draft_logits"][:, :, :V], host["draft_hidden"], host["p_hidden"], host["p_logit"],
+                     host["w1"], host["b1"], host["w2"], host["b2"], n, n_bs)
+    ws = P.VerifyWorkspace(n_bs, cfg.n_q_heads, cfg.n_kv_heads)
+    st = StagedRequests(req)
+    dev = {k: (v.cuda().contiguous() if torch.is_tensor(v) else v) for k, v in d.items()}
+    pred = torch.full((n_bs, 15), 7.0, dtype=torch.float32, device="cuda")
+    feat = torch.full((n_bs, 1735), 7.0, dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        P.predict_scores(ws, st.n_live, dev["draft_logits"], V, dev["draft_hidden"], dev["p_hidden"],
+                         dev["p_logit"], dev["w1"], dev["b1"], dev["w2"], dev["b2"], pred, feat)
+        torch.cuda.synchronize()
+    f, ref = feat.cpu().numpy().astype(np.float64), exp["features"]
+    assert (f[n:] == 0).all() and (pred.cpu().numpy()[n:] == 0).all()
+    conf = f[:n, :270].reshape(n, 15, 18)
+    rconf = ref[:, :270].reshape(n, 15, 18)
+    np.testing.assert_array_equal(conf[:, :, 0], rconf[:, :, 0].astype(np.float32))
+    np.testing.assert_allclose(conf[:, :, 1:16], rconf[:, :, 1:16], rtol=1e-6, atol=1e-6)
+    np.testing.assert_allclose(conf[:, :, 16:], rconf[:, :, 16:], rtol=0, atol=2e-4)
+    np.testing.assert_allclose(f[:n, 270:1230], ref[:, 270:1230], rtol=1e-4, atol=1e-4)
+    np.testing.assert_allclose(f[:n, 1230:1710], ref[:, 1230:1710], rtol=2e-3, atol=4e-3)
+    np.testing.assert_array_equal(f[:n, 1710:], ref[:, 1710:])
+    got = pred.cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(got[:n], exp["pred_logits"][:n], rtol=3e-3, atol=3e-3)
+    # the allocation the device builds from its own predLogits
+    P.alloc_verify(ws, st.n_live, pred, st.draft, st.ctx_len, st.block_table, req["num_pages"],
+                   scores_are_logits=True)
+    torch.cuda.synchronize()
+    assert ws.status() == 0
+    scores = np.zeros((n_bs, 15), dtype=np.float32)
+    scores[:n] = pred.cpu().numpy()[:n]
+    want = OA.dvl_alloc(n_bs, n, scores, req["draft_tokens"], req["ctx_len"], req["block_table"],
+                        logits_mode=True)
+    assert_alloc_equal({k: ws.field(k).cpu().numpy() for k in ALLOC_FIELDS}, want)
+    return exp
+
+
+@pytest.mark.parametrize("n_bs,n,vocab,hidden_dim", [
+    (4, 3, 1003, 64),         # odd vocabulary (scalar projection loads), one row group with dead rows
+    (20, 17, 50000, 512),     # several row groups and chunks, a ragged last chunk
+    (64, 64, 4096, 128),      # largest capacity
+    (2, 1, 16, 8),            # smallest legal shapes
+])
+def test_predictor_small_shapes(n_bs, n, vocab, hidden_dim):
+    import paper_2609_37532_b200 as P
+    cfg = small_variant(CONFIGS["tiny"], vocab=vocab, n=n, seed=71 + n_bs)
+    _case(P, cfg, n_bs, hidden_dim)
+
+
+def test_predictor_constant_offset_changes_only_the_top_logit():
+    """Property at any size: a common offset on a request's logits leaves everything but the
+    18-strided top-logit entries unchanged (within rounding)."""
+    import paper_2609_37532_b200 as P
+    cfg = small_variant(CONFIGS["tiny"], vocab=8192, n=4, seed=77)
+    req = make_requests(cfg, n_bs=4)
+    d = {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in make_predictor_inputs(req, 64).items()}
+    ws = P.VerifyWorkspace(4, cfg.n_q_heads, cfg.n_kv_heads)
+    st = StagedRequests(req)
+    outs = []
+    for off in (0.0, 16.0):
+        pred = torch.zeros((4, 15), dtype=torch.float32, device="cuda")
+        feat = torch.zeros((4, 1735), dtype=torch.float32, device="cuda")
+        P.predict_scores(ws, st.n_live, d["draft_logits"] + off, 8192, d["draft_hidden"], d["p_hidden"],
+                         d["p_logit"], d["w1"], d["b1"], d["w2"], d["b2"], pred, feat)
+        torch.cuda.synchronize()
+        outs.append(feat.cpu().numpy())
+    a, b = outs
+    top = np.zeros(1735, dtype=bool); top[0:270:18] = True
+    np.testing.assert_allclose(b[:, top], a[:, top] + 16.0, rtol=1e-6)
+    np.testing.assert_allclose(b[:, ~top], a[:, ~top], rtol=2e-3, atol=4e-3)
+
+
+def test_predictor_full_size_qwen3_8b():
+    """B = 32, vocabulary 151936, drafter hidden size 4096: 480 logit rows, 292 MB."""
+    import paper_2609_37532_b200 as P
+    cfg = CONFIGS["qwen3_8b_step"]
+    _case(P, cfg, cfg.n, 4096, gen_device="cuda")
+
+
+def test_predictor_rejects_bad_shapes():
+    import paper_2609_37532_b200 as P
+    ws = P.VerifyWorkspace(2, 32, 8)
+    z = torch.zeros((2, 15, 1002), dtype=torch.float32, device="cuda")      # ld % 4 != 0
+    h = torch.zeros((2, 15, 64), dtype=torch.bfloat16, device="cuda")
+    ph = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    pl = torch.zeros((32, 1002), dtype=torch.bfloat16, device="cuda")
+    w1 = torch.zeros((64, 1735), device="cuda"); b1 = torch.zeros(64, device="cuda")
+    w2 = torch.zeros((15, 64), device="cuda"); b2 = torch.zeros(15, device="cuda")
+    out = torch.zeros((2, 15), device="cuda")
+    nl = torch.ones(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(RuntimeError):
+        P.predict_scores(ws, nl, z, 1002, h, ph, pl, w1, b1, w2, b2, out)
