@@ -28,7 +28,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 from dscale_inputs import (CONFIGS, make_kv_layer, make_lm_head_unpacked, make_logits_unpacked,  # noqa: E402
-                           make_q_unpacked, make_requests, rows_to_packed, small_variant)
+                           make_predictor_inputs, make_q_unpacked, make_requests, rows_to_packed, small_variant)
 
 SCALE = 1.0 / float(np.sqrt(128.0))
 METRIC = "verified_tokens_per_s"
@@ -384,6 +384,29 @@ def run_ours(args, rank, world, local_rank):
                   "frac_of_bf16_peak": lm_flops / (lm_ms * 1e-3) / 1e12 / measured_bf16_peak()}
             del w_lm, h_lm, lg
 
+        # the predictor front end (three launches) on seeded drafter outputs
+        pred = None
+        if args.pred_hidden > 0:
+            pin = make_predictor_inputs(req, args.pred_hidden, device=str(dev))
+            pl_out = torch.zeros((n_bs, 15), dtype=torch.float32, device=dev)
+
+            def do_pred():
+                P.predict_scores(ws, d_n_live, pin["draft_logits"], cfg.vocab, pin["draft_hidden"], pin["p_hidden"],
+                                 pin["p_logit"], pin["w1"], pin["b1"], pin["w2"], pin["b2"], pl_out)
+            for _ in range(3):
+                do_pred()
+            ea.record(stream)
+            for _ in range(args.steps):
+                do_pred()
+            eb.record(stream)
+            barrier()
+            pred_ms = ea.elapsed_time(eb) / args.steps
+            pred_bytes = 15 * n * cfg.vocab * 4 + 32 * cfg.vocab * 2 + 15 * n * args.pred_hidden * 2
+            pred = {"us": pred_ms * 1e3, "hidden": args.pred_hidden, "bytes": pred_bytes,
+                    "gbs": pred_bytes / (pred_ms * 1e-3) / 1e9,
+                    "frac_of_hbm_peak": pred_bytes / (pred_ms * 1e-3) / 1e9 / measured_peak()[0]}
+            del pin
+
         # ---- timed region 3: end to end through the host-buffer C ABI call ----
         hs = P.HostStep(ws, req["max_pages"], req["num_pages"], layers, logits, cfg.vocab, SCALE)
         hs.h_n_live[0] = n
@@ -436,7 +459,7 @@ def run_ours(args, rank, world, local_rank):
                          "bytes_per_launch": per_layer_b, "us_per_launch": attn_ms * 1e3,
                          "traffic": recorded_traffic(cfg.name)},
             "accept_us": accept_ms * 1e3, "accept_sampling_us": sampling_ms * 1e3,
-            "lm_head_accept": lm,
+            "lm_head_accept": lm, "predict_scores": pred,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": hs.h2d_bytes,
                     "d2h_bytes_per_step": hs.d2h_bytes, "ms_per_step": 1e3 * e2e_s / args.steps,
                     "api": "dscale_verify_step_host (pinned host inputs/outputs, KV/Q/logits resident)"},
@@ -493,6 +516,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--lm-hidden", type=int, default=4096,
                     help="hidden size of the fused LM-head figure (0 skips it)")
+    ap.add_argument("--pred-hidden", type=int, default=4096,
+                    help="drafter hidden size of the predictor front-end figure (0 skips it)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-padded", action="store_true", help="skip the padded comparison kernel")
     ap.add_argument("--cpu-layers", type=int, default=0,

@@ -280,7 +280,7 @@ int dscale_lm_head_accept(void* ws, int n_bs, const void* hidden, const void* we
  *   features_out  nullable fp32 [n_bs][1735] out (rows >= N set to 0)
  * fp32 arithmetic; the logit projection rounds (z - z[0]) to tf32 for the tensor
  * cores (the centring is applied afterwards, exactly).  All pointers are device
- * pointers owned by the caller, 16-byte aligned.  Three launches on `stream`, no
+ * pointers owned by the caller, 16-byte aligned.  Four launches on `stream`, no
  * allocation, no synchronisation; scratch lives in ws.  vocab >= 16.
  * Errors: DSCALE_ERR_INVALID_ARG (null / misaligned), DSCALE_ERR_UNSUPPORTED
  * (shape rules above), DSCALE_ERR_WORKSPACE (unknown ws).

@@ -1,6 +1,6 @@
 // Acceptance-predictor front end: drafter logits and hidden states -> 1735
 // features -> 1735-64-15 perceptron -> predLogits ("Acceptance predictor"
-// paragraph, Eq. 4 and Eq. 5).  Three launches:
+// paragraph, Eq. 4 and Eq. 5).  Four launches:
 //
 //  pred_stream_kernel    the only pass over the drafter logits (15 N rows x V fp32,
 //                        292 MB at N = 32: an HBM stream).  A CTA of 16 warps owns
@@ -21,14 +21,15 @@
 //                        One record per (row, chunk) goes to the workspace.
 //  pred_features_kernel  per request: merges the chunk records into the 18
 //                        confidence values and the centred logit projection per
-//                        position, computes the 64 x H hidden-state projection,
-//                        appends the batch context.
+//                        position, appends the batch context.
+//  pred_hidden_kernel    the 64 x H hidden-state projection of all rows (bf16 MMAs).
 //  pred_mlp_kernel       per request: relu(W1 f + b1), W2 h + b2.
 #include <cfloat>
 #include <climits>
 #include <cuda_bf16.h>
 
 #include "kernels.cuh"
+#include "tc_ptx.cuh"
 
 namespace dscale {
 
@@ -38,7 +39,6 @@ constexpr int kRowsPerCta = 16;                 // = warps per CTA = k steps per
 constexpr int kStreamThreads = kRowsPerCta * 32;
 constexpr int kSub = 128;                       // columns per sub-tile: one float4 per lane
 constexpr int kStride = kSub + 4;               // shared-memory row stride in floats (conflict-free fragments)
-constexpr int kStreamSmem = 2 * (kRowsPerCta + kPredLog) * kStride * 4;   // 50,688 bytes
 
 struct StreamArgs {
   const float* logits;      // [15 n_bs][ld]
@@ -51,6 +51,7 @@ struct StreamArgs {
   float* rowsum;            // [chunks][32]
   int chunks;
   int chunk_len;            // multiple of kSub
+  int* status;              // workspace status word
 };
 
 __device__ __forceinline__ float to_tf32(float x) {
@@ -89,11 +90,55 @@ __device__ __forceinline__ void top16_offer(float& tv, float& tau, float z, int 
   }
 }
 
-__global__ void __launch_bounds__(kStreamThreads, 2) pred_stream_kernel(StreamArgs a) {
-  extern __shared__ __align__(16) float stream_smem[];
-  float (*zs)[kRowsPerCta][kStride] = reinterpret_cast<float (*)[kRowsPerCta][kStride]>(stream_smem);
-  float (*ps)[kPredLog][kStride] =
-      reinterpret_cast<float (*)[kPredLog][kStride]>(stream_smem + 2 * kRowsPerCta * kStride);
+// Shared-memory ring: per stage the 16 rows' sub-tile of raw fp32 logits (four TMA
+// boxes of 32 columns x 16 rows) and the 32 x 128 bf16 tile of the projection
+// matrix (two boxes of 64 columns x 32 rows), 128-byte swizzle, six copy
+// instructions per 16 KB stage issued by six lanes of warp 0.  (One bulk copy
+// per row was tried first: 48 small copies per stage cap the copy engine at
+// about 1 TB/s.)  Bytes in flight per SM are set by the ring depth, not by
+// registers.
+constexpr int kStages = 6;
+constexpr int kZStage = kRowsPerCta * kSub * 4;           // 8192 bytes: 4 boxes of 2 KB
+constexpr int kPStage = kPredLog * kSub * 2;              // 8192 bytes: 2 boxes of 4 KB
+constexpr int kOffP = kStages * kZStage;
+constexpr int kOffPivot = kOffP + kStages * kPStage;
+constexpr int kOffBar = kOffPivot + kRowsPerCta * 4;
+constexpr int kOffAbort = kOffBar + 2 * kStages * 8;       // full[kStages], empty[kStages]
+constexpr int kStreamSmem = kOffAbort + 16 + 1024;        // + slack to align the ring to 1024 bytes
+
+// byte offset of logit (row r, column c) inside a stage's swizzled logit boxes
+__device__ __forceinline__ uint32_t z_off(int r, int c) {
+  return (uint32_t)((c >> 5) * 2048 + r * 128 + ((((c & 31) >> 2) ^ (r & 7)) << 4) + ((c & 3) << 2));
+}
+// byte offset of projection weight (output j, column c) inside a stage's swizzled boxes
+__device__ __forceinline__ uint32_t p_off(int j, int c) {
+  return (uint32_t)((c >> 6) * 4096 + j * 128 + ((((c & 63) >> 3) ^ (j & 7)) << 4) + ((c & 7) << 1));
+}
+__device__ __forceinline__ void tma_box_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+__global__ void __launch_bounds__(kStreamThreads, 2)
+pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const __grid_constant__ CUtensorMap tm_p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t sbase = (raw + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (sbase - raw);
+  float* pivots = reinterpret_cast<float*>(smem + kOffPivot);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + kOffAbort);
+  auto zs = [&](int st, int r, int c) -> float* {
+    return reinterpret_cast<float*>(smem + st * kZStage + z_off(r, c));
+  };
+  auto psm = [&](int st, int j, int c) -> unsigned short* {
+    return reinterpret_cast<unsigned short*>(smem + kOffP + st * kPStage + p_off(j, c));
+  };
+  auto full = [&](int st) { return sbase + kOffBar + 8u * st; };
+  auto empty = [&](int st) { return sbase + kOffBar + 8u * (kStages + st); };
+
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int n = *a.n_live;
   n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
@@ -107,105 +152,166 @@ __global__ void __launch_bounds__(kStreamThreads, 2) pred_stream_kernel(StreamAr
   const int n_sub = (col_hi - col_lo + kSub - 1) / kSub;
 
   const bool live = row0 + warp < live_rows;
-  const int row = live ? row0 + warp : row0;          // dead rows re-read a live one; results dropped
-  const float* zrow = a.logits + (size_t)row * a.ld;
-  const float pivot = zrow[0];
+  const bool p_vec = (a.vocab & 7) == 0;               // projection rows 16-byte aligned: TMA
+  const int pj = tid >> 4, pq = tid & 15;               // scalar staging and row sums: (output, 8 columns)
 
-  // projection-matrix staging: thread -> (output j, 8 columns)
-  const int pj = tid >> 4, pq = tid & 15;
-  const __nv_bfloat16* prow = a.p_logit + (size_t)pj * a.vocab;
-  const bool p_vec = (a.vocab & 7) == 0;               // 16-byte loads stay aligned
-  float p_rowsum = 0.f;
-
-  auto load_z = [&](int s) -> float4 {
-    const int c = col_lo + s * kSub + 4 * lane;
-    float4 z = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-    if (c < col_hi) {
-      z = ldg_stream4(zrow + c);                        // rows are padded to ld % 4 == 0
-      if (c + 1 >= col_hi) z.y = -INFINITY;
-      if (c + 2 >= col_hi) z.z = -INFINITY;
-      if (c + 3 >= col_hi) z.w = -INFINITY;
+  if (tid == 0) {
+    // full: the copy engine's transaction count, plus one arrival per warp when the warps
+    // stage the projection tile by hand; empty: every warp has finished with the stage
+    for (int st = 0; st < kStages; ++st) {
+      mbar_init(full(st), p_vec ? 1 : 1 + kRowsPerCta);
+      mbar_init(empty(st), kRowsPerCta);
     }
-    return z;
-  };
-  auto load_p = [&](int s, float (&pv)[8]) {
-    const int c = col_lo + s * kSub + 8 * pq;
-    if (p_vec && c + 8 <= col_hi) {
-      const uint4 u = __ldg(reinterpret_cast<const uint4*>(prow + c));
-      const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    s_abort[0] = 0; s_abort[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_z) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_p) : "memory");
+  }
+  if (lane == 0) pivots[warp] = live ? a.logits[(size_t)(row0 + warp) * a.ld] : 0.f;
+  __syncthreads();
+
+  // Fill stage st with sub-tile v; the caller has made sure the stage is free.  Warp 0
+  // issues the copies (columns beyond the vocabulary and rows beyond the tensor arrive
+  // as zeros).  With an odd vocabulary the projection rows are not 16-byte aligned:
+  // every warp then stores its two rows by hand and arrives on the full barrier.
+  auto fill = [&](int v, int st) {
+    const int c = col_lo + v * kSub;
+    if (warp == 0) {
+      if (lane == 0) mbar_expect_tx(full(st), kZStage + (p_vec ? kPStage : 0));
+      __syncwarp();
+      if (lane < 4) tma_box_2d(sbase + st * kZStage + lane * 2048, &tm_z, full(st), c + 32 * lane, row0);
+      else if (lane < 6 && p_vec)
+        tma_box_2d(sbase + kOffP + st * kPStage + (lane - 4) * 4096, &tm_p, full(st), c + 64 * (lane - 4), 0);
+    }
+    if (!p_vec) {
 #pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        pv[2 * x] = __uint_as_float(w[x] << 16);
-        pv[2 * x + 1] = __uint_as_float(w[x] & 0xffff0000u);
+      for (int x = 0; x < 8; ++x) {
+        const int e = lane + 32 * x, j = 2 * warp + (e >> 7), cc = e & 127;       // two rows of 128 columns
+        *psm(st, j, cc) = c + cc < col_hi ? __bfloat16_as_ushort(a.p_logit[(size_t)j * a.vocab + c + cc])
+                                          : (unsigned short)0;
       }
-    } else {
-#pragma unroll
-      for (int x = 0; x < 8; ++x) pv[x] = c + x < col_hi ? __bfloat162float(prow[c + x]) : 0.f;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full(st));
     }
   };
 
   float m = -INFINITY, s_sum = 0.f, t_sum = 0.f, z_sum = 0.f;
   float tv = -INFINITY, tau = -INFINITY;
+  float p_rowsum = 0.f;
   float d[4][4];
 #pragma unroll
   for (int x = 0; x < 4; ++x) d[x][0] = d[x][1] = d[x][2] = d[x][3] = 0.f;
   const int g = lane >> 2, t = lane & 3;
 
-  float4 z_next = load_z(0);
-  float p_next[8];
-  load_p(0, p_next);
-  for (int s = 0; s < n_sub; ++s) {
-    const int b = s & 1;
-    const float4 z = z_next;
-    // stage this sub-tile: logits minus pivot as tf32 (0 beyond the chunk), projection tile as fp32
-    {
-      float4 c4;
-      c4.x = z.x == -INFINITY ? 0.f : to_tf32(z.x - pivot);
-      c4.y = z.y == -INFINITY ? 0.f : to_tf32(z.y - pivot);
-      c4.z = z.z == -INFINITY ? 0.f : to_tf32(z.z - pivot);
-      c4.w = z.w == -INFINITY ? 0.f : to_tf32(z.w - pivot);
-      *reinterpret_cast<float4*>(&zs[b][warp][4 * lane]) = c4;
-      *reinterpret_cast<float4*>(&ps[b][pj][8 * pq]) = make_float4(p_next[0], p_next[1], p_next[2], p_next[3]);
-      *reinterpret_cast<float4*>(&ps[b][pj][8 * pq + 4]) = make_float4(p_next[4], p_next[5], p_next[6], p_next[7]);
-#pragma unroll
-      for (int x = 0; x < 8; ++x) p_rowsum += p_next[x];
-    }
-    if (s + 1 < n_sub) { z_next = load_z(s + 1); load_p(s + 1, p_next); }
-    __syncthreads();
+  const int pre = n_sub < kStages ? n_sub : kStages;
+  for (int v = 0; v < pre; ++v) fill(v, v);
+  const float piv_lo = pivots[g], piv_hi = pivots[g + 8];
+  // Per-thread constants of the loop.  The k slots (t, t + 4) of this warp's MMA step
+  // stand for columns 8 warp + 2t and + 2t + 1 (the same permutation for both
+  // operands), so a fragment is one 8-byte logit load per row and one 4-byte load of
+  // a bf16 pair per output tile.  Columns beyond the vocabulary need no mask here:
+  // the projection tile is zero there.
+  const uint32_t zo_lo = z_off(g, 8 * warp + 2 * t), zo_hi = z_off(g + 8, 8 * warp + 2 * t);
+  const uint32_t po = kOffP + p_off(g, 8 * warp + 2 * t);           // + 1024 per output tile
+  const uint32_t so = z_off(warp, 4 * lane);                         // this lane's four logits of row `warp`
+  const uint32_t ro = kOffP + p_off(pj, 8 * pq);                     // row sums: eight weights of output pj
 
-    // ---- row statistics on the exact fp32 values
-    {
-      const float zl = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
-      if (zl > m) {
-        const float r = __expf(m - zl);                 // m = -inf gives 0
-        s_sum *= r; t_sum *= r; m = zl;
-      }
-      const float zz[4] = {z.x, z.y, z.z, z.w};
+  int st = 0;
+  uint32_t parity = 0;
+  bool ok = true;
+  int u = 0;
+  for (; u < n_sub; ++u) {
+    ok = mbar_wait(full(st), parity, s_abort);
+    if (ok) {
+      const unsigned char* zst = smem + st * kZStage;
+      const unsigned char* pst = smem + st * kPStage;
+      // ---- row statistics on the exact fp32 values
+      if (live) {
+        float4 z = *reinterpret_cast<const float4*>(zst + so);
+        const int c = col_lo + u * kSub + 4 * lane;
+        if (c + 3 >= col_hi) {                              // ragged end of the vocabulary
+          if (c >= col_hi) z.x = -INFINITY;
+          if (c + 1 >= col_hi) z.y = -INFINITY;
+          if (c + 2 >= col_hi) z.z = -INFINITY;
+          z.w = -INFINITY;
+        }
+        const float zl = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
+        if (zl > m) {
+          const float r = __expf(m - zl);                   // m = -inf gives 0
+          s_sum *= r; t_sum *= r; m = zl;
+        }
+        const float zz[4] = {z.x, z.y, z.z, z.w};
+        if (c + 3 < col_hi) {
 #pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        if (zz[x] != -INFINITY) {
-          const float e = __expf(zz[x] - m);
-          s_sum += e; t_sum = fmaf(e, zz[x], t_sum); z_sum += zz[x];
+          for (int x = 0; x < 4; ++x) {
+            const float e = __expf(zz[x] - m);
+            s_sum += e; t_sum = fmaf(e, zz[x], t_sum); z_sum += zz[x];
+          }
+        } else {
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            if (zz[x] != -INFINITY) {
+              const float e = __expf(zz[x] - m);
+              s_sum += e; t_sum = fmaf(e, zz[x], t_sum); z_sum += zz[x];
+            }
+          }
+        }
+        if (__any_sync(0xffffffffu, zl > tau)) {            // rare once the list has warmed up
+          top16_offer(tv, tau, z.x, lane);
+          top16_offer(tv, tau, z.y, lane);
+          top16_offer(tv, tau, z.z, lane);
+          top16_offer(tv, tau, z.w, lane);
         }
       }
-      top16_offer(tv, tau, z.x, lane);
-      top16_offer(tv, tau, z.y, lane);
-      top16_offer(tv, tau, z.z, lane);
-      top16_offer(tv, tau, z.w, lane);
-    }
-    // ---- this warp's k step of the logit projection: columns 8 warp .. 8 warp + 7
-    {
-      const int k0 = 8 * warp;
-      uint32_t af[4];
-      af[0] = __float_as_uint(zs[b][g][k0 + t]);
-      af[1] = __float_as_uint(zs[b][g + 8][k0 + t]);
-      af[2] = __float_as_uint(zs[b][g][k0 + t + 4]);
-      af[3] = __float_as_uint(zs[b][g + 8][k0 + t + 4]);
+      // ---- this warp's k step of the logit projection
+      {
+        const float2 zlo = *reinterpret_cast<const float2*>(zst + zo_lo);
+        const float2 zhi = *reinterpret_cast<const float2*>(zst + zo_hi);
+        uint32_t af[4];
+        af[0] = __float_as_uint(to_tf32(zlo.x - piv_lo));
+        af[1] = __float_as_uint(to_tf32(zhi.x - piv_hi));
+        af[2] = __float_as_uint(to_tf32(zlo.y - piv_lo));
+        af[3] = __float_as_uint(to_tf32(zhi.y - piv_hi));
 #pragma unroll
-      for (int nt = 0; nt < 4; ++nt)
-        mma_tf32(d[nt], af, __float_as_uint(ps[b][8 * nt + g][k0 + t]),
-                 __float_as_uint(ps[b][8 * nt + g][k0 + t + 4]));
+        for (int nt = 0; nt < 4; ++nt) {
+          const uint32_t w = *reinterpret_cast<const uint32_t*>(pst + po + 1024 * nt);
+          mma_tf32(d[nt], af, w << 16, w & 0xffff0000u);
+        }
+      }
+      // ---- row sums of the projection matrix (first row group only)
+      if (blockIdx.y == 0) {
+        const uint4 w = *reinterpret_cast<const uint4*>(pst + ro);
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+          p_rowsum += __uint_as_float(ww[x] << 16) + __uint_as_float(ww[x] & 0xffff0000u);
+      }
     }
+    if (!ok) break;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty(st));                  // this warp is done with the stage
+    // refill the PREVIOUS stage (one iteration late, so that nobody waits for the slowest warp)
+    if (u >= 1 && u - 1 + kStages < n_sub) {
+      const int sp = st == 0 ? kStages - 1 : st - 1;
+      const uint32_t pp = st == 0 ? parity ^ 1 : parity;    // phase of the sub-tile u - 1 in that stage
+      if (warp == 0 || !p_vec) {
+        ok = mbar_wait(empty(sp), pp, s_abort);
+        if (!ok) break;
+        fill(u - 1 + kStages, sp);
+      }
+    }
+    if (++st == kStages) { st = 0; parity ^= 1; }
+  }
+  __syncthreads();
+  if (*s_abort) {
+    // Some wait ran out.  Let the copies already issued land before the shared memory is
+    // released (bounded), flag the status word, and leave.
+    if (tid == 0) {
+      for (int x = 0; x < kStages; ++x) { mbar_wait(full(x), 0, s_abort + 1); mbar_wait(full(x), 1, s_abort + 1); }
+      atomicOr(a.status, 8 /*TIMEOUT*/);
+    }
+    __syncthreads();
+    return;
   }
 
   // ---- row statistics: merge the 32 lanes
@@ -221,15 +327,14 @@ __global__ void __launch_bounds__(kStreamThreads, 2) pred_stream_kernel(StreamAr
     t_sum = t_sum * r1 + t2 * r2;
     m = mm;
   }
-  float* rec = a.part + ((size_t)(row0 + warp) * a.chunks + chunk) * kPredRec;
   if (live) {
+    float* rec = a.part + ((size_t)(row0 + warp) * a.chunks + chunk) * kPredRec;
     if (lane < 16) rec[lane] = tv;
     if (lane == 0) { rec[16] = m; rec[17] = s_sum; rec[18] = t_sum; rec[19] = z_sum; }
   }
-  // ---- projection: sum the 16 warps' k slices through shared memory
-  __syncthreads();
-  float* red = &ps[0][0][0];                            // 16 x 512 floats fit the two projection buffers
-  static_assert(2 * kPredLog * kStride >= kRowsPerCta * 512, "reduction buffer");
+  // ---- projection: sum the 16 warps' k slices through shared memory (the ring is idle now)
+  float* red = reinterpret_cast<float*>(smem);
+  static_assert(kStages * kZStage >= kRowsPerCta * 512 * 4, "reduction buffer");
 #pragma unroll
   for (int nt = 0; nt < 4; ++nt) {
     red[warp * 512 + g * 32 + 8 * nt + 2 * t] = d[nt][0];
@@ -246,7 +351,6 @@ __global__ void __launch_bounds__(kStreamThreads, 2) pred_stream_kernel(StreamAr
     if (row0 + r < live_rows)
       a.part[((size_t)(row0 + r) * a.chunks + chunk) * kPredRec + 20 + j] = acc;
   }
-  // ---- row sums of the projection matrix over this chunk (first row group only)
   if (blockIdx.y == 0) {
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) p_rowsum += __shfl_xor_sync(0xffffffffu, p_rowsum, o);
@@ -271,7 +375,6 @@ struct FeatArgs {
 };
 
 constexpr int kFeatThreads = 256;
-constexpr int kHidPerBlock = 16;   // hidden-projection outputs per block: grid.y = 1 + 64 / 16
 
 __global__ void __launch_bounds__(kFeatThreads) pred_features_kernel(FeatArgs a) {
   const int i = blockIdx.x;
@@ -281,7 +384,7 @@ __global__ void __launch_bounds__(kFeatThreads) pred_features_kernel(FeatArgs a)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   float* f = a.feat + (size_t)i * kPredFeatures;
 
-  if (blockIdx.y == 0) {
+  {
     // ---- confidence values and centred logit projection, one warp per position
     for (int p = warp; p < kPredPos; p += kFeatThreads / 32) {
       const int row = i * kPredPos + p;
@@ -328,45 +431,69 @@ __global__ void __launch_bounds__(kFeatThreads) pred_features_kernel(FeatArgs a)
     }
     if (warp == 0 && lane < kPredCtx)
       f[kPredFeatures - kPredCtx + lane] = lane == 0 ? (float)n : (lane == 3 ? 1.f : 0.f);
-  } else {
-    // ---- hidden-state projection: kHidPerBlock outputs x 15 positions, two outputs per warp
-    const int H = a.hidden_dim;
-    const __nv_bfloat16* hbase = a.hidden + (size_t)i * kPredPos * H;
-    for (int jj = warp; jj < kHidPerBlock; jj += kFeatThreads / 32) {
-      const int j = (blockIdx.y - 1) * kHidPerBlock + jj;
-      const __nv_bfloat16* prow = a.p_hidden + (size_t)j * H;
-      float acc[kPredPos];
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Hidden-state projection: [15 N rows x H] . [H x 64], a small dense contraction
+// (0.25 GFLOP at N = 32, H = 4096) on warp-level bf16 MMAs.  A CTA owns 16 rows;
+// its 8 warps split H in blocks of 32 and are summed through shared memory.  The
+// k slots of the MMA are a permutation of the 32 columns of a block (the same
+// one for both operands), so every fragment is one 16-byte load.
+constexpr int kHidThreads = 256;
+
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__global__ void __launch_bounds__(kHidThreads) pred_hidden_kernel(FeatArgs a) {
+  __shared__ float red[kHidThreads / 32][16 * kPredHid];
+  int n = *a.n_live;
+  n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
+  const int live_rows = kPredPos * n;
+  const int row0 = blockIdx.x * 16;
+  if (row0 >= live_rows) return;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int H = a.hidden_dim;
+  const int r_lo = min(row0 + g, live_rows - 1), r_hi = min(row0 + g + 8, live_rows - 1);
+  const __nv_bfloat16* h_lo = a.hidden + (size_t)r_lo * H;
+  const __nv_bfloat16* h_hi = a.hidden + (size_t)r_hi * H;
+  float d[8][4];
 #pragma unroll
-      for (int p = 0; p < kPredPos; ++p) acc[p] = 0.f;
-      for (int c = 8 * lane; c < H; c += 256) {         // hidden_dim % 8 == 0
-        const uint4 pu = __ldg(reinterpret_cast<const uint4*>(prow + c));
-        const uint32_t pw[4] = {pu.x, pu.y, pu.z, pu.w};
-        float pf[8];
+  for (int x = 0; x < 8; ++x) d[x][0] = d[x][1] = d[x][2] = d[x][3] = 0.f;
+  const uint4 zero4 = make_uint4(0, 0, 0, 0);
+  for (int kb = warp * 32; kb < H; kb += 32 * (kHidThreads / 32)) {
+    const int c = kb + 8 * t;                              // hidden_dim % 8 == 0: a chunk is in or out
+    const bool in = c < H;
+    const uint4 alo = in ? __ldg(reinterpret_cast<const uint4*>(h_lo + c)) : zero4;
+    const uint4 ahi = in ? __ldg(reinterpret_cast<const uint4*>(h_hi + c)) : zero4;
 #pragma unroll
-        for (int x = 0; x < 4; ++x) {
-          pf[2 * x] = __uint_as_float(pw[x] << 16);
-          pf[2 * x + 1] = __uint_as_float(pw[x] & 0xffff0000u);
-        }
+    for (int nt = 0; nt < 8; ++nt) {
+      const uint4 b = in ? __ldg(reinterpret_cast<const uint4*>(a.p_hidden + (size_t)(8 * nt + g) * H + c)) : zero4;
+      mma_bf16(d[nt], alo.x, ahi.x, alo.y, ahi.y, b.x, b.y);
+      mma_bf16(d[nt], alo.z, ahi.z, alo.w, ahi.w, b.z, b.w);
+    }
+  }
 #pragma unroll
-        for (int p = 0; p < kPredPos; ++p) {
-          const uint4 hu = __ldg(reinterpret_cast<const uint4*>(hbase + (size_t)p * H + c));
-          const uint32_t hw[4] = {hu.x, hu.y, hu.z, hu.w};
+  for (int nt = 0; nt < 8; ++nt) {
+    red[warp][g * kPredHid + 8 * nt + 2 * t] = d[nt][0];
+    red[warp][g * kPredHid + 8 * nt + 2 * t + 1] = d[nt][1];
+    red[warp][(g + 8) * kPredHid + 8 * nt + 2 * t] = d[nt][2];
+    red[warp][(g + 8) * kPredHid + 8 * nt + 2 * t + 1] = d[nt][3];
+  }
+  __syncthreads();
+  for (int x = tid; x < 16 * kPredHid; x += kHidThreads) {
+    float acc = 0.f;
 #pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            acc[p] = fmaf(pf[2 * x], __uint_as_float(hw[x] << 16), acc[p]);
-            acc[p] = fmaf(pf[2 * x + 1], __uint_as_float(hw[x] & 0xffff0000u), acc[p]);
-          }
-        }
-      }
-#pragma unroll
-      for (int p = 0; p < kPredPos; ++p) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc[p] += __shfl_xor_sync(0xffffffffu, acc[p], o);
-      }
-      if (lane == 0) {
-#pragma unroll
-        for (int p = 0; p < kPredPos; ++p) f[kPredPos * kPredConf + p * kPredHid + j] = acc[p];
-      }
+    for (int w = 0; w < kHidThreads / 32; ++w) acc += red[w][x];
+    const int row = row0 + (x >> 6), j = x & 63;
+    if (row < live_rows) {
+      const int i = row / kPredPos, p = row - i * kPredPos;
+      a.feat[(size_t)i * kPredFeatures + kPredPos * kPredConf + p * kPredHid + j] = acc;
     }
   }
 }
@@ -403,13 +530,23 @@ __global__ void __launch_bounds__(256) pred_mlp_kernel(MlpArgs a) {
     if (a.features_out) a.features_out[(size_t)i * kPredFeatures + x] = v;
   }
   __syncthreads();
-  for (int j = warp; j < kPredMlp; j += 8) {
-    const float* w = a.w1 + (size_t)j * kPredFeatures;
-    float acc = 0.f;
-    for (int x = lane; x < kPredFeatures; x += 32) acc = fmaf(w[x], sf[x], acc);
+  {
+    // warp w computes hidden units 8 w .. 8 w + 7 together: eight independent weight streams
+    const float* w = a.w1 + (size_t)(8 * warp) * kPredFeatures;
+    float acc[8];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) sh[j] = fmaxf(acc + a.b1[j], 0.f);
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    for (int x = lane; x < kPredFeatures; x += 32) {
+      const float fx = sf[x];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[j] = fmaf(__ldg(w + (size_t)j * kPredFeatures + x), fx, acc[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+      if (lane == 0) sh[8 * warp + j] = fmaxf(acc[j] + a.b1[8 * warp + j], 0.f);
+    }
   }
   __syncthreads();
   for (int o = warp; o < kPredPos; o += 8) {
@@ -422,6 +559,38 @@ __global__ void __launch_bounds__(256) pred_mlp_kernel(MlpArgs a) {
 }
 
 }  // namespace
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn pred_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+// row-major [rows][inner] matrix with a row pitch, box [box_rows][box_inner], 128-byte swizzle
+static bool pred_encode(CUtensorMap* out, CUtensorMapDataType dt, int elem, const void* ptr, uint64_t inner,
+                        uint64_t rows, uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows) {
+  EncodeTiledFn enc = pred_encode_fn();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {box_inner, box_rows};
+  cuuint32_t es[2] = {1, 1};
+  (void)elem;
+  return enc(out, dt, 2, const_cast<void*>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 cudaError_t predictor_prepare() {
   return cudaFuncSetAttribute(pred_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
@@ -448,14 +617,29 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   const int row_groups = (kPredPos * p.n_bs + kRowsPerCta - 1) / kRowsPerCta;
 
   StreamArgs sa{p.draft_logits, p.ld, p.vocab, p.n_live, p.n_bs,
-                reinterpret_cast<const __nv_bfloat16*>(p.p_logit), part, rowsum, chunks, chunk_len};
-  pred_stream_kernel<<<dim3(chunks, row_groups), kStreamThreads, kStreamSmem, stream>>>(sa);
+                reinterpret_cast<const __nv_bfloat16*>(p.p_logit), part, rowsum, chunks, chunk_len,
+                ws_ptr<int>(p.ws, L.hdr) + H_STATUS};
+  CUtensorMap tz, tp;
+  if (!pred_encode(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.draft_logits, (uint64_t)p.vocab,
+                   (uint64_t)kPredPos * p.n_bs, (uint64_t)p.ld * 4, 32, kRowsPerCta))
+    return cudaErrorNotSupported;
+  if ((p.vocab & 7) == 0) {
+    if (!pred_encode(&tp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.p_logit, (uint64_t)p.vocab, kPredLog,
+                     (uint64_t)p.vocab * 2, 64, kPredLog))
+      return cudaErrorNotSupported;
+  } else {
+    tp = tz;                                            // never used: odd vocabularies stage the matrix by hand
+  }
+  pred_stream_kernel<<<dim3(chunks, row_groups), kStreamThreads, kStreamSmem, stream>>>(sa, tz, tp);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   FeatArgs fa{p.draft_logits, p.ld, p.vocab, p.n_live, p.n_bs,
               reinterpret_cast<const __nv_bfloat16*>(p.draft_hidden), p.hidden_dim,
               reinterpret_cast<const __nv_bfloat16*>(p.p_hidden), part, rowsum, chunks, feat};
-  pred_features_kernel<<<dim3(p.n_bs, 1 + kPredHid / kHidPerBlock), kFeatThreads, 0, stream>>>(fa);
+  pred_features_kernel<<<p.n_bs, kFeatThreads, 0, stream>>>(fa);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  pred_hidden_kernel<<<row_groups, kHidThreads, 0, stream>>>(fa);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   MlpArgs ma{p.n_live, p.n_bs, feat, p.w1, p.b1, p.w2, p.b2, p.pred_logits, p.features_out};
