@@ -35,8 +35,9 @@ namespace dscale {
 
 namespace {
 
-constexpr int kRowsPerCta = 16;                 // = warps per CTA = k steps per sub-tile
-constexpr int kStreamThreads = kRowsPerCta * 32;
+constexpr int kWarps = 16;                      // warps per CTA = k steps of 8 per sub-tile
+constexpr int kRowsPerCta = 2 * kWarps;         // each warp streams two rows
+constexpr int kStreamThreads = kWarps * 32;
 constexpr int kSub = 128;                       // columns per sub-tile: one float4 per lane
 constexpr int kStride = kSub + 4;               // shared-memory row stride in floats (conflict-free fragments)
 
@@ -90,49 +91,94 @@ __device__ __forceinline__ void top16_offer(float& tv, float& tau, float z, int 
   }
 }
 
-// Shared-memory ring: per stage the 16 rows' sub-tile of raw fp32 logits (four TMA
-// boxes of 32 columns x 16 rows) and the 32 x 128 bf16 tile of the projection
-// matrix (two boxes of 64 columns x 32 rows), 128-byte swizzle, six copy
-// instructions per 16 KB stage issued by six lanes of warp 0.  (One bulk copy
-// per row was tried first: 48 small copies per stage cap the copy engine at
-// about 1 TB/s.)  Bytes in flight per SM are set by the ring depth, not by
-// registers.
+// Shared-memory ring: per stage the 32 rows' sub-tile of raw fp32 logits (16 KB) and
+// the 32 x 128 bf16 tile of the projection matrix (8 KB), filled by per-thread
+// 16-byte cp.async copies (every thread: one piece of each of its warp's two rows,
+// one piece of the tile) that arrive on the stage's mbarrier when they land.  Bytes
+// in flight per SM are set by the ring depth, not by registers.  (Tried first: one
+// bulk copy per row, then TMA boxes of 2-4 KB; both were bound by the copy
+// engine's per-instruction cost, about 100-200 cycles per SM whatever the box
+// size.)  The layout inside a stage is the 128-byte XOR swizzle, so that the MMA
+// fragment loads are free of bank conflicts.  One CTA per SM, one wave.
 constexpr int kStages = 6;
-constexpr int kZStage = kRowsPerCta * kSub * 4;           // 8192 bytes: 4 boxes of 2 KB
-constexpr int kPStage = kPredLog * kSub * 2;              // 8192 bytes: 2 boxes of 4 KB
+constexpr int kZStage = kRowsPerCta * kSub * 4;           // 16 KB: 4 column groups x 32 rows x 128 bytes
+constexpr int kPStage = kPredLog * kSub * 2;              // 8 KB: 2 column groups x 32 outputs x 128 bytes
 constexpr int kOffP = kStages * kZStage;
 constexpr int kOffPivot = kOffP + kStages * kPStage;
 constexpr int kOffBar = kOffPivot + kRowsPerCta * 4;
 constexpr int kOffAbort = kOffBar + 2 * kStages * 8;       // full[kStages], empty[kStages]
 constexpr int kStreamSmem = kOffAbort + 16 + 1024;        // + slack to align the ring to 1024 bytes
 
-// byte offset of logit (row r, column c) inside a stage's swizzled logit boxes
+// byte offset of logit (row r, column c) inside a stage's swizzled logit tile
 __device__ __forceinline__ uint32_t z_off(int r, int c) {
-  return (uint32_t)((c >> 5) * 2048 + r * 128 + ((((c & 31) >> 2) ^ (r & 7)) << 4) + ((c & 3) << 2));
+  return (uint32_t)((c >> 5) * (kRowsPerCta * 128) + r * 128 + ((((c & 31) >> 2) ^ (r & 7)) << 4) + ((c & 3) << 2));
 }
-// byte offset of projection weight (output j, column c) inside a stage's swizzled boxes
+// byte offset of projection weight (output j, column c) inside a stage's swizzled tile
 __device__ __forceinline__ uint32_t p_off(int j, int c) {
   return (uint32_t)((c >> 6) * 4096 + j * 128 + ((((c & 63) >> 3) ^ (j & 7)) << 4) + ((c & 7) << 1));
 }
-__device__ __forceinline__ void tma_box_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-      "[%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
-      : "memory");
+// 16-byte asynchronous copy global -> shared; bytes beyond `valid` are written as zeros
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int valid) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid) : "memory");
+}
+// arrive on the barrier once all earlier cp.async of this thread have landed
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__global__ void __launch_bounds__(kStreamThreads, 2)
-pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const __grid_constant__ CUtensorMap tm_p) {
+// running statistics of one logit row in one lane
+struct RowStat {
+  float m2, s, t, zsum;      // m2 = running max times log2(e)
+  float tv, tau;             // sorted top-16 (lane = rank) and the current 16th value
+};
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ void row_update(RowStat& r, float4 z, int c, int col_hi, int lane) {
+  const bool ragged = c + 3 >= col_hi;
+  if (ragged) {                                             // end of the vocabulary
+    if (c >= col_hi) z.x = -INFINITY;
+    if (c + 1 >= col_hi) z.y = -INFINITY;
+    if (c + 2 >= col_hi) z.z = -INFINITY;
+    z.w = -INFINITY;
+  }
+  const float zl = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
+  const float zl2 = zl * kLog2e;
+  if (zl2 > r.m2) {
+    const float f = ex2(r.m2 - zl2);                        // m2 = -inf gives 0
+    r.s *= f; r.t *= f; r.m2 = zl2;
+  }
+  const float zz[4] = {z.x, z.y, z.z, z.w};
+  if (!ragged) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const float e = ex2(fmaf(zz[x], kLog2e, -r.m2));
+      r.s += e; r.t = fmaf(e, zz[x], r.t); r.zsum += zz[x];
+    }
+  } else {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      if (zz[x] != -INFINITY) {
+        const float e = exp2f(fmaf(zz[x], kLog2e, -r.m2));
+        r.s += e; r.t = fmaf(e, zz[x], r.t); r.zsum += zz[x];
+      }
+    }
+  }
+  if (__any_sync(0xffffffffu, zl > r.tau)) {                // rare once the list has warmed up
+    top16_offer(r.tv, r.tau, z.x, lane);
+    top16_offer(r.tv, r.tau, z.y, lane);
+    top16_offer(r.tv, r.tau, z.z, lane);
+    top16_offer(r.tv, r.tau, z.w, lane);
+  }
+}
+
+__global__ void __launch_bounds__(kStreamThreads, 1)
+pred_stream_kernel(StreamArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t sbase = (raw + 1023u) & ~1023u;
   unsigned char* smem = smem_raw + (sbase - raw);
   float* pivots = reinterpret_cast<float*>(smem + kOffPivot);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + kOffAbort);
-  auto zs = [&](int st, int r, int c) -> float* {
-    return reinterpret_cast<float*>(smem + st * kZStage + z_off(r, c));
-  };
   auto psm = [&](int st, int j, int c) -> unsigned short* {
     return reinterpret_cast<unsigned short*>(smem + kOffP + st * kPStage + p_off(j, c));
   };
@@ -151,39 +197,45 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
   if (col_lo >= col_hi) return;
   const int n_sub = (col_hi - col_lo + kSub - 1) / kSub;
 
-  const bool live = row0 + warp < live_rows;
-  const bool p_vec = (a.vocab & 7) == 0;               // projection rows 16-byte aligned: TMA
-  const int pj = tid >> 4, pq = tid & 15;               // scalar staging and row sums: (output, 8 columns)
+  // warp w owns rows w and w + 16 of the CTA's 32 (one in each 16-row MMA tile)
+  const int my_row[2] = {row0 + warp, row0 + warp + kWarps};
+  const bool live[2] = {my_row[0] < live_rows, my_row[1] < live_rows};
+  const bool p_vec = (a.vocab & 7) == 0;               // projection rows 16-byte aligned
+  const int pj = tid >> 4, pq = tid & 15;               // projection tile piece: (output, 8 columns)
 
   if (tid == 0) {
-    // full: the copy engine's transaction count, plus one arrival per warp when the warps
-    // stage the projection tile by hand; empty: every warp has finished with the stage
+    // full: every thread arrives when its copies of the stage have landed (plus one
+    // arrival per warp when the warps store the projection tile by hand);
+    // empty: every warp has finished with the stage
     for (int st = 0; st < kStages; ++st) {
-      mbar_init(full(st), p_vec ? 1 : 1 + kRowsPerCta);
-      mbar_init(empty(st), kRowsPerCta);
+      mbar_init(full(st), kStreamThreads + (p_vec ? 0 : kWarps));
+      mbar_init(empty(st), kWarps);
     }
     s_abort[0] = 0; s_abort[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_z) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_p) : "memory");
   }
-  if (lane == 0) pivots[warp] = live ? a.logits[(size_t)(row0 + warp) * a.ld] : 0.f;
+  if (lane < 2) pivots[warp + kWarps * lane] = live[lane] ? a.logits[(size_t)my_row[lane] * a.ld] : 0.f;
   __syncthreads();
 
-  // Fill stage st with sub-tile v; the caller has made sure the stage is free.  Warp 0
-  // issues the copies (columns beyond the vocabulary and rows beyond the tensor arrive
-  // as zeros).  With an odd vocabulary the projection rows are not 16-byte aligned:
-  // every warp then stores its two rows by hand and arrives on the full barrier.
+  // Fill stage st with sub-tile v; the caller has made sure the stage is free.  Ragged
+  // ends are zero-filled by the copy.  With an odd vocabulary the projection rows are
+  // not 16-byte aligned: every warp then stores its two projection rows by hand.
+  const float* zsrc0 = a.logits + (size_t)(live[0] ? my_row[0] : row0) * a.ld + 4 * lane;
+  const float* zsrc1 = a.logits + (size_t)(live[1] ? my_row[1] : row0) * a.ld + 4 * lane;
+  const __nv_bfloat16* psrc = a.p_logit + (size_t)pj * a.vocab + 8 * pq;
+  const uint32_t so0 = z_off(warp, 4 * lane), so1 = z_off(warp + kWarps, 4 * lane);
+  const uint32_t ro = kOffP + p_off(pj, 8 * pq);
   auto fill = [&](int v, int st) {
     const int c = col_lo + v * kSub;
-    if (warp == 0) {
-      if (lane == 0) mbar_expect_tx(full(st), kZStage + (p_vec ? kPStage : 0));
-      __syncwarp();
-      if (lane < 4) tma_box_2d(sbase + st * kZStage + lane * 2048, &tm_z, full(st), c + 32 * lane, row0);
-      else if (lane < 6 && p_vec)
-        tma_box_2d(sbase + kOffP + st * kPStage + (lane - 4) * 4096, &tm_p, full(st), c + 64 * (lane - 4), 0);
-    }
-    if (!p_vec) {
+    const int zleft = (a.vocab - (c + 4 * lane)) * 4;                 // zeros beyond the vocabulary
+    const int zvalid = zleft >= 16 ? 16 : (zleft > 0 ? zleft : 0);
+    if (live[0]) cp_async16(sbase + st * kZStage + so0, zvalid ? zsrc0 + c : a.logits, zvalid);
+    if (live[1]) cp_async16(sbase + st * kZStage + so1, zvalid ? zsrc1 + c : a.logits, zvalid);
+    if (p_vec) {
+      const int left = (a.vocab - (c + 8 * pq)) * 2;
+      const int valid = left >= 16 ? 16 : (left > 0 ? left : 0);
+      cp_async16(sbase + st * kPStage + ro, valid ? psrc + c : a.p_logit, valid);
+    } else {
 #pragma unroll
       for (int x = 0; x < 8; ++x) {
         const int e = lane + 32 * x, j = 2 * warp + (e >> 7), cc = e & 127;       // two rows of 128 columns
@@ -193,161 +245,141 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
       __syncwarp();
       if (lane == 0) mbar_arrive(full(st));
     }
+    cp_async_arrive(full(st));
   };
 
-  float m = -INFINITY, s_sum = 0.f, t_sum = 0.f, z_sum = 0.f;
-  float tv = -INFINITY, tau = -INFINITY;
-  float p_rowsum = 0.f;
-  float d[4][4];
+  RowStat rs[2];
 #pragma unroll
-  for (int x = 0; x < 4; ++x) d[x][0] = d[x][1] = d[x][2] = d[x][3] = 0.f;
+  for (int x = 0; x < 2; ++x) {
+    rs[x].m2 = -INFINITY; rs[x].s = 0.f; rs[x].t = 0.f; rs[x].zsum = 0.f; rs[x].tv = -INFINITY; rs[x].tau = -INFINITY;
+  }
+  float p_rowsum = 0.f;
+  float d[2][4][4];
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+#pragma unroll
+    for (int x = 0; x < 4; ++x) d[h][x][0] = d[h][x][1] = d[h][x][2] = d[h][x][3] = 0.f;
   const int g = lane >> 2, t = lane & 3;
 
   const int pre = n_sub < kStages ? n_sub : kStages;
   for (int v = 0; v < pre; ++v) fill(v, v);
-  const float piv_lo = pivots[g], piv_hi = pivots[g + 8];
   // Per-thread constants of the loop.  The k slots (t, t + 4) of this warp's MMA step
   // stand for columns 8 warp + 2t and + 2t + 1 (the same permutation for both
   // operands), so a fragment is one 8-byte logit load per row and one 4-byte load of
   // a bf16 pair per output tile.  Columns beyond the vocabulary need no mask here:
-  // the projection tile is zero there.
-  const uint32_t zo_lo = z_off(g, 8 * warp + 2 * t), zo_hi = z_off(g + 8, 8 * warp + 2 * t);
+  // both tiles are zero there.
+  float piv[4];
+  uint32_t zo[4];
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {                             // rows g, g + 8, g + 16, g + 24
+    piv[x] = pivots[g + 8 * x];
+    zo[x] = z_off(g + 8 * x, 8 * warp + 2 * t);
+  }
   const uint32_t po = kOffP + p_off(g, 8 * warp + 2 * t);           // + 1024 per output tile
-  const uint32_t so = z_off(warp, 4 * lane);                         // this lane's four logits of row `warp`
-  const uint32_t ro = kOffP + p_off(pj, 8 * pq);                     // row sums: eight weights of output pj
 
   int st = 0;
   uint32_t parity = 0;
   bool ok = true;
-  int u = 0;
-  for (; u < n_sub; ++u) {
+  for (int u = 0; u < n_sub; ++u) {
     ok = mbar_wait(full(st), parity, s_abort);
-    if (ok) {
-      const unsigned char* zst = smem + st * kZStage;
-      const unsigned char* pst = smem + st * kPStage;
-      // ---- row statistics on the exact fp32 values
-      if (live) {
-        float4 z = *reinterpret_cast<const float4*>(zst + so);
-        const int c = col_lo + u * kSub + 4 * lane;
-        if (c + 3 >= col_hi) {                              // ragged end of the vocabulary
-          if (c >= col_hi) z.x = -INFINITY;
-          if (c + 1 >= col_hi) z.y = -INFINITY;
-          if (c + 2 >= col_hi) z.z = -INFINITY;
-          z.w = -INFINITY;
-        }
-        const float zl = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
-        if (zl > m) {
-          const float r = __expf(m - zl);                   // m = -inf gives 0
-          s_sum *= r; t_sum *= r; m = zl;
-        }
-        const float zz[4] = {z.x, z.y, z.z, z.w};
-        if (c + 3 < col_hi) {
+    if (!ok) break;
+    const unsigned char* zst = smem + st * kZStage;
+    const unsigned char* pst = smem + st * kPStage;
+    // ---- row statistics on the exact fp32 values
+    const int c = col_lo + u * kSub + 4 * lane;
+    if (live[0]) row_update(rs[0], *reinterpret_cast<const float4*>(zst + so0), c, col_hi, lane);
+    if (live[1]) row_update(rs[1], *reinterpret_cast<const float4*>(zst + so1), c, col_hi, lane);
+    // ---- this warp's k step of the logit projection, both 16-row tiles
+    {
+      uint32_t bw[4];
 #pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const float e = __expf(zz[x] - m);
-            s_sum += e; t_sum = fmaf(e, zz[x], t_sum); z_sum += zz[x];
-          }
-        } else {
+      for (int nt = 0; nt < 4; ++nt) bw[nt] = *reinterpret_cast<const uint32_t*>(pst + po + 1024 * nt);
 #pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            if (zz[x] != -INFINITY) {
-              const float e = __expf(zz[x] - m);
-              s_sum += e; t_sum = fmaf(e, zz[x], t_sum); z_sum += zz[x];
-            }
-          }
-        }
-        if (__any_sync(0xffffffffu, zl > tau)) {            // rare once the list has warmed up
-          top16_offer(tv, tau, z.x, lane);
-          top16_offer(tv, tau, z.y, lane);
-          top16_offer(tv, tau, z.z, lane);
-          top16_offer(tv, tau, z.w, lane);
-        }
-      }
-      // ---- this warp's k step of the logit projection
-      {
-        const float2 zlo = *reinterpret_cast<const float2*>(zst + zo_lo);
-        const float2 zhi = *reinterpret_cast<const float2*>(zst + zo_hi);
+      for (int h = 0; h < 2; ++h) {
+        const float2 zlo = *reinterpret_cast<const float2*>(zst + zo[2 * h]);
+        const float2 zhi = *reinterpret_cast<const float2*>(zst + zo[2 * h + 1]);
         uint32_t af[4];
-        af[0] = __float_as_uint(to_tf32(zlo.x - piv_lo));
-        af[1] = __float_as_uint(to_tf32(zhi.x - piv_hi));
-        af[2] = __float_as_uint(to_tf32(zlo.y - piv_lo));
-        af[3] = __float_as_uint(to_tf32(zhi.y - piv_hi));
+        af[0] = __float_as_uint(to_tf32(zlo.x - piv[2 * h]));
+        af[1] = __float_as_uint(to_tf32(zhi.x - piv[2 * h + 1]));
+        af[2] = __float_as_uint(to_tf32(zlo.y - piv[2 * h]));
+        af[3] = __float_as_uint(to_tf32(zhi.y - piv[2 * h + 1]));
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
-          const uint32_t w = *reinterpret_cast<const uint32_t*>(pst + po + 1024 * nt);
-          mma_tf32(d[nt], af, w << 16, w & 0xffff0000u);
-        }
-      }
-      // ---- row sums of the projection matrix (first row group only)
-      if (blockIdx.y == 0) {
-        const uint4 w = *reinterpret_cast<const uint4*>(pst + ro);
-        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-        for (int x = 0; x < 4; ++x)
-          p_rowsum += __uint_as_float(ww[x] << 16) + __uint_as_float(ww[x] & 0xffff0000u);
+        for (int nt = 0; nt < 4; ++nt) mma_tf32(d[h][nt], af, bw[nt] << 16, bw[nt] & 0xffff0000u);
       }
     }
-    if (!ok) break;
+    // ---- row sums of the projection matrix (first row group only)
+    if (blockIdx.y == 0) {
+      const uint4 w = *reinterpret_cast<const uint4*>(pst + ro);
+      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int x = 0; x < 4; ++x)
+        p_rowsum += __uint_as_float(ww[x] << 16) + __uint_as_float(ww[x] & 0xffff0000u);
+    }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty(st));                  // this warp is done with the stage
     // refill the PREVIOUS stage (one iteration late, so that nobody waits for the slowest warp)
     if (u >= 1 && u - 1 + kStages < n_sub) {
       const int sp = st == 0 ? kStages - 1 : st - 1;
       const uint32_t pp = st == 0 ? parity ^ 1 : parity;    // phase of the sub-tile u - 1 in that stage
-      if (warp == 0 || !p_vec) {
-        ok = mbar_wait(empty(sp), pp, s_abort);
-        if (!ok) break;
-        fill(u - 1 + kStages, sp);
-      }
+      ok = mbar_wait(empty(sp), pp, s_abort);
+      if (!ok) break;
+      fill(u - 1 + kStages, sp);
     }
     if (++st == kStages) { st = 0; parity ^= 1; }
   }
   __syncthreads();
   if (*s_abort) {
-    // Some wait ran out.  Let the copies already issued land before the shared memory is
-    // released (bounded), flag the status word, and leave.
-    if (tid == 0) {
-      for (int x = 0; x < kStages; ++x) { mbar_wait(full(x), 0, s_abort + 1); mbar_wait(full(x), 1, s_abort + 1); }
-      atomicOr(a.status, 8 /*TIMEOUT*/);
-    }
+    // Some wait ran out.  Let this thread's copies land before the shared memory is
+    // released, flag the status word, and leave.
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    if (tid == 0) atomicOr(a.status, 8 /*TIMEOUT*/);
     __syncthreads();
     return;
   }
 
-  // ---- row statistics: merge the 32 lanes
+  // ---- row statistics: merge the 32 lanes, write the records
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
-    const float s2 = __shfl_xor_sync(0xffffffffu, s_sum, o);
-    const float t2 = __shfl_xor_sync(0xffffffffu, t_sum, o);
-    z_sum += __shfl_xor_sync(0xffffffffu, z_sum, o);
-    const float mm = fmaxf(m, m2);
-    const float r1 = m == -INFINITY ? 0.f : __expf(m - mm), r2 = m2 == -INFINITY ? 0.f : __expf(m2 - mm);
-    s_sum = s_sum * r1 + s2 * r2;
-    t_sum = t_sum * r1 + t2 * r2;
-    m = mm;
-  }
-  if (live) {
-    float* rec = a.part + ((size_t)(row0 + warp) * a.chunks + chunk) * kPredRec;
-    if (lane < 16) rec[lane] = tv;
-    if (lane == 0) { rec[16] = m; rec[17] = s_sum; rec[18] = t_sum; rec[19] = z_sum; }
+  for (int x = 0; x < 2; ++x) {
+    float m2 = rs[x].m2, s_sum = rs[x].s, t_sum = rs[x].t, z_sum = rs[x].zsum;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float mo = __shfl_xor_sync(0xffffffffu, m2, o);
+      const float s2 = __shfl_xor_sync(0xffffffffu, s_sum, o);
+      const float t2 = __shfl_xor_sync(0xffffffffu, t_sum, o);
+      z_sum += __shfl_xor_sync(0xffffffffu, z_sum, o);
+      const float mm = fmaxf(m2, mo);
+      const float r1 = m2 == -INFINITY ? 0.f : exp2f(m2 - mm), r2 = mo == -INFINITY ? 0.f : exp2f(mo - mm);
+      s_sum = s_sum * r1 + s2 * r2;
+      t_sum = t_sum * r1 + t2 * r2;
+      m2 = mm;
+    }
+    if (live[x]) {
+      float* rec = a.part + ((size_t)my_row[x] * a.chunks + chunk) * kPredRec;
+      if (lane < 16) rec[lane] = rs[x].tv;
+      if (lane == 0) { rec[16] = m2 / kLog2e; rec[17] = s_sum; rec[18] = t_sum; rec[19] = z_sum; }
+    }
   }
   // ---- projection: sum the 16 warps' k slices through shared memory (the ring is idle now)
   float* red = reinterpret_cast<float*>(smem);
-  static_assert(kStages * kZStage >= kRowsPerCta * 512 * 4, "reduction buffer");
+  constexpr int kTile = kRowsPerCta * kPredLog;             // 1024 projections per CTA
+  static_assert(kStages * kZStage >= kWarps * kTile * 4, "reduction buffer");
 #pragma unroll
-  for (int nt = 0; nt < 4; ++nt) {
-    red[warp * 512 + g * 32 + 8 * nt + 2 * t] = d[nt][0];
-    red[warp * 512 + g * 32 + 8 * nt + 2 * t + 1] = d[nt][1];
-    red[warp * 512 + (g + 8) * 32 + 8 * nt + 2 * t] = d[nt][2];
-    red[warp * 512 + (g + 8) * 32 + 8 * nt + 2 * t + 1] = d[nt][3];
+  for (int h = 0; h < 2; ++h) {
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      float* q = red + warp * kTile + (16 * h + g) * kPredLog + 8 * nt + 2 * t;
+      q[0] = d[h][nt][0]; q[1] = d[h][nt][1];
+      q[8 * kPredLog] = d[h][nt][2]; q[8 * kPredLog + 1] = d[h][nt][3];
+    }
   }
   __syncthreads();
-  {
+#pragma unroll
+  for (int y = 0; y < kTile / kStreamThreads; ++y) {
+    const int e = tid + y * kStreamThreads;
     float acc = 0.f;
 #pragma unroll
-    for (int w = 0; w < kRowsPerCta; ++w) acc += red[w * 512 + tid];
-    const int r = tid >> 5, j = tid & 31;
+    for (int w = 0; w < kWarps; ++w) acc += red[w * kTile + e];
+    const int r = e >> 5, j = e & 31;
     if (row0 + r < live_rows)
       a.part[((size_t)(row0 + r) * a.chunks + chunk) * kPredRec + 20 + j] = acc;
   }
@@ -560,45 +592,13 @@ __global__ void __launch_bounds__(256) pred_mlp_kernel(MlpArgs a) {
 
 }  // namespace
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static EncodeTiledFn pred_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-// row-major [rows][inner] matrix with a row pitch, box [box_rows][box_inner], 128-byte swizzle
-static bool pred_encode(CUtensorMap* out, CUtensorMapDataType dt, int elem, const void* ptr, uint64_t inner,
-                        uint64_t rows, uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows) {
-  EncodeTiledFn enc = pred_encode_fn();
-  if (!enc) return false;
-  cuuint64_t dims[2] = {inner, rows};
-  cuuint64_t strides[1] = {pitch_bytes};
-  cuuint32_t box[2] = {box_inner, box_rows};
-  cuuint32_t es[2] = {1, 1};
-  (void)elem;
-  return enc(out, dt, 2, const_cast<void*>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 cudaError_t predictor_prepare() {
   return cudaFuncSetAttribute(pred_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
 }
 
 int predictor_chunks(int n_bs, int vocab, int num_ctas, int* chunk_len_out) {
   const int row_groups = (kPredPos * n_bs + kRowsPerCta - 1) / kRowsPerCta;
-  int chunks = (3 * num_ctas + row_groups - 1) / row_groups;      // about three CTAs per SM
+  int chunks = num_ctas / row_groups;                             // one CTA per SM, a single wave
   chunks = chunks < 1 ? 1 : (chunks > kPredMaxChunks ? kPredMaxChunks : chunks);
   int chunk_len = (vocab + chunks - 1) / chunks;
   chunk_len = (chunk_len + kSub - 1) / kSub * kSub;
@@ -619,18 +619,7 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   StreamArgs sa{p.draft_logits, p.ld, p.vocab, p.n_live, p.n_bs,
                 reinterpret_cast<const __nv_bfloat16*>(p.p_logit), part, rowsum, chunks, chunk_len,
                 ws_ptr<int>(p.ws, L.hdr) + H_STATUS};
-  CUtensorMap tz, tp;
-  if (!pred_encode(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.draft_logits, (uint64_t)p.vocab,
-                   (uint64_t)kPredPos * p.n_bs, (uint64_t)p.ld * 4, 32, kRowsPerCta))
-    return cudaErrorNotSupported;
-  if ((p.vocab & 7) == 0) {
-    if (!pred_encode(&tp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.p_logit, (uint64_t)p.vocab, kPredLog,
-                     (uint64_t)p.vocab * 2, 64, kPredLog))
-      return cudaErrorNotSupported;
-  } else {
-    tp = tz;                                            // never used: odd vocabularies stage the matrix by hand
-  }
-  pred_stream_kernel<<<dim3(chunks, row_groups), kStreamThreads, kStreamSmem, stream>>>(sa, tz, tp);
+  pred_stream_kernel<<<dim3(chunks, row_groups), kStreamThreads, kStreamSmem, stream>>>(sa);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   FeatArgs fa{p.draft_logits, p.ld, p.vocab, p.n_live, p.n_bs,
@@ -639,7 +628,7 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   pred_features_kernel<<<p.n_bs, kFeatThreads, 0, stream>>>(fa);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  pred_hidden_kernel<<<row_groups, kHidThreads, 0, stream>>>(fa);
+  pred_hidden_kernel<<<(kPredPos * p.n_bs + 15) / 16, kHidThreads, 0, stream>>>(fa);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   MlpArgs ma{p.n_live, p.n_bs, feat, p.w1, p.b1, p.w2, p.b2, p.pred_logits, p.features_out};
