@@ -37,7 +37,7 @@ namespace {
 
 constexpr int kWarps = 16;                      // warps per CTA = k steps of 8 per sub-tile
 constexpr int kRowsPerCta = 2 * kWarps;         // each warp streams two rows
-constexpr int kStreamThreads = kWarps * 32;
+constexpr int kStreamThreads = (kWarps + 1) * 32;   // + one copy warp
 constexpr int kSub = 128;                       // columns per sub-tile: one float4 per lane
 constexpr int kStride = kSub + 4;               // shared-memory row stride in floats (conflict-free fragments)
 
@@ -92,15 +92,16 @@ __device__ __forceinline__ void top16_offer(float& tv, float& tau, float z, int 
 }
 
 // Shared-memory ring: per stage the 32 rows' sub-tile of raw fp32 logits (16 KB) and
-// the 32 x 128 bf16 tile of the projection matrix (8 KB), filled by per-thread
-// 16-byte cp.async copies (every thread: one piece of each of its warp's two rows,
-// one piece of the tile) that arrive on the stage's mbarrier when they land.  Bytes
-// in flight per SM are set by the ring depth, not by registers.  (Tried first: one
-// bulk copy per row, then TMA boxes of 2-4 KB; both were bound by the copy
-// engine's per-instruction cost, about 100-200 cycles per SM whatever the box
-// size.)  The layout inside a stage is the 128-byte XOR swizzle, so that the MMA
-// fragment loads are free of bank conflicts.  One CTA per SM, one wave.
-constexpr int kStages = 6;
+// the 32 x 128 bf16 tile of the projection matrix (8 KB), filled by a copy warp with
+// six TMA boxes per stage; the 16 compute warps only wait for "full" and signal
+// "empty", so a warp that is busy inserting into its top-16 list holds nobody up
+// until the ring runs dry.  (Tried on the way: every warp copying its own rows and
+// waiting for the slowest warp once per stage; one bulk copy per row, which is
+// bound by the copy engine's per-instruction cost; per-thread cp.async issued by a
+// single warp, which is bound by that warp's instruction issue.)  The layout
+// inside a stage is the 128-byte XOR swizzle, so that the MMA fragment loads are
+// free of bank conflicts.  One CTA per SM, one wave.
+constexpr int kStages = 8;
 constexpr int kZStage = kRowsPerCta * kSub * 4;           // 16 KB: 4 column groups x 32 rows x 128 bytes
 constexpr int kPStage = kPredLog * kSub * 2;              // 8 KB: 2 column groups x 32 outputs x 128 bytes
 constexpr int kOffP = kStages * kZStage;
@@ -116,6 +117,13 @@ __device__ __forceinline__ uint32_t z_off(int r, int c) {
 // byte offset of projection weight (output j, column c) inside a stage's swizzled tile
 __device__ __forceinline__ uint32_t p_off(int j, int c) {
   return (uint32_t)((c >> 6) * 4096 + j * 128 + ((((c & 63) >> 3) ^ (j & 7)) << 4) + ((c & 7) << 1));
+}
+__device__ __forceinline__ void tma_box_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
 }
 // 16-byte asynchronous copy global -> shared; bytes beyond `valid` are written as zeros
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int valid) {
@@ -172,7 +180,7 @@ __device__ __forceinline__ void row_update(RowStat& r, float4 z, int c, int col_
 }
 
 __global__ void __launch_bounds__(kStreamThreads, 1)
-pred_stream_kernel(StreamArgs a) {
+pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const __grid_constant__ CUtensorMap tm_p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t sbase = (raw + 1023u) & ~1023u;
@@ -199,54 +207,63 @@ pred_stream_kernel(StreamArgs a) {
 
   // warp w owns rows w and w + 16 of the CTA's 32 (one in each 16-row MMA tile)
   const int my_row[2] = {row0 + warp, row0 + warp + kWarps};
-  const bool live[2] = {my_row[0] < live_rows, my_row[1] < live_rows};
+  const bool live[2] = {warp < kWarps && my_row[0] < live_rows, warp < kWarps && my_row[1] < live_rows};
   const bool p_vec = (a.vocab & 7) == 0;               // projection rows 16-byte aligned
   const int pj = tid >> 4, pq = tid & 15;               // projection tile piece: (output, 8 columns)
 
   if (tid == 0) {
-    // full: every thread arrives when its copies of the stage have landed (plus one
-    // arrival per warp when the warps store the projection tile by hand);
-    // empty: every warp has finished with the stage
+    // full: the copy warp's expect-tx arrival (plus one arrival when that warp stores the
+    // projection tile by hand); empty: every compute warp has finished with the stage
     for (int st = 0; st < kStages; ++st) {
-      mbar_init(full(st), kStreamThreads + (p_vec ? 0 : kWarps));
+      mbar_init(full(st), p_vec ? 1 : 2);
       mbar_init(empty(st), kWarps);
     }
     s_abort[0] = 0; s_abort[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (lane < 2) pivots[warp + kWarps * lane] = live[lane] ? a.logits[(size_t)my_row[lane] * a.ld] : 0.f;
+  if (warp < kWarps && lane < 2) pivots[warp + kWarps * lane] = live[lane] ? a.logits[(size_t)my_row[lane] * a.ld] : 0.f;
   __syncthreads();
 
-  // Fill stage st with sub-tile v; the caller has made sure the stage is free.  Ragged
-  // ends are zero-filled by the copy.  With an odd vocabulary the projection rows are
-  // not 16-byte aligned: every warp then stores its two projection rows by hand.
-  const float* zsrc0 = a.logits + (size_t)(live[0] ? my_row[0] : row0) * a.ld + 4 * lane;
-  const float* zsrc1 = a.logits + (size_t)(live[1] ? my_row[1] : row0) * a.ld + 4 * lane;
-  const __nv_bfloat16* psrc = a.p_logit + (size_t)pj * a.vocab + 8 * pq;
-  const uint32_t so0 = z_off(warp, 4 * lane), so1 = z_off(warp + kWarps, 4 * lane);
-  const uint32_t ro = kOffP + p_off(pj, 8 * pq);
-  auto fill = [&](int v, int st) {
-    const int c = col_lo + v * kSub;
-    const int zleft = (a.vocab - (c + 4 * lane)) * 4;                 // zeros beyond the vocabulary
-    const int zvalid = zleft >= 16 ? 16 : (zleft > 0 ? zleft : 0);
-    if (live[0]) cp_async16(sbase + st * kZStage + so0, zvalid ? zsrc0 + c : a.logits, zvalid);
-    if (live[1]) cp_async16(sbase + st * kZStage + so1, zvalid ? zsrc1 + c : a.logits, zvalid);
-    if (p_vec) {
-      const int left = (a.vocab - (c + 8 * pq)) * 2;
-      const int valid = left >= 16 ? 16 : (left > 0 ? left : 0);
-      cp_async16(sbase + st * kPStage + ro, valid ? psrc + c : a.p_logit, valid);
-    } else {
-#pragma unroll
-      for (int x = 0; x < 8; ++x) {
-        const int e = lane + 32 * x, j = 2 * warp + (e >> 7), cc = e & 127;       // two rows of 128 columns
-        *psm(st, j, cc) = c + cc < col_hi ? __bfloat16_as_ushort(a.p_logit[(size_t)j * a.vocab + c + cc])
-                                          : (unsigned short)0;
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(full(st));
+  if (warp == kWarps) {
+    // ===================================================== copy warp
+    // Per 24 KB stage six TMA boxes, one lane each: four of 32 columns x 32 rows of
+    // logits, two of 64 columns x 32 outputs of the projection matrix (128-byte
+    // swizzle; columns beyond the vocabulary and rows beyond the tensor arrive as
+    // zeros).  With an odd vocabulary the projection rows are not 16-byte aligned and
+    // are stored by hand (slow, but such vocabularies are not the case to tune for).
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_z) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_p) : "memory");
     }
-    cp_async_arrive(full(st));
-  };
+    int st = 0;
+    uint32_t parity = 1;                                    // a fresh barrier passes a wait on parity 1
+    bool ok = true;
+    for (int v = 0; v < n_sub && ok; ++v) {
+      ok = mbar_wait(empty(st), parity, s_abort);
+      if (!ok) break;
+      const int c = col_lo + v * kSub;
+      if (lane == 0) mbar_expect_tx(full(st), kZStage + (p_vec ? kPStage : 0));
+      __syncwarp();
+      if (lane < 4) tma_box_2d(sbase + st * kZStage + lane * (kRowsPerCta * 128), &tm_z, full(st), c + 32 * lane, row0);
+      else if (lane < 6 && p_vec)
+        tma_box_2d(sbase + kOffP + st * kPStage + (lane - 4) * 4096, &tm_p, full(st), c + 64 * (lane - 4), 0);
+      if (!p_vec) {
+        for (int e = lane; e < kPredLog * kSub; e += 32) {
+          const int j = e >> 7, cc = e & 127;
+          *psm(st, j, cc) = c + cc < col_hi ? __bfloat16_as_ushort(a.p_logit[(size_t)j * a.vocab + c + cc])
+                                            : (unsigned short)0;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full(st));
+      }
+      if (++st == kStages) { st = 0; parity ^= 1; }
+    }
+    // every stage issued has been, or will be, waited for by the compute warps; on an
+    // aborted run wait (bounded) for the copies in flight before the CTA may exit
+    if (!ok) {
+      for (int x = 0; x < kStages; ++x) { mbar_wait(full(x), 0, s_abort + 1); mbar_wait(full(x), 1, s_abort + 1); }
+    }
+  }
 
   RowStat rs[2];
 #pragma unroll
@@ -261,8 +278,6 @@ pred_stream_kernel(StreamArgs a) {
     for (int x = 0; x < 4; ++x) d[h][x][0] = d[h][x][1] = d[h][x][2] = d[h][x][3] = 0.f;
   const int g = lane >> 2, t = lane & 3;
 
-  const int pre = n_sub < kStages ? n_sub : kStages;
-  for (int v = 0; v < pre; ++v) fill(v, v);
   // Per-thread constants of the loop.  The k slots (t, t + 4) of this warp's MMA step
   // stand for columns 8 warp + 2t and + 2t + 1 (the same permutation for both
   // operands), so a fragment is one 8-byte logit load per row and one 4-byte load of
@@ -273,14 +288,16 @@ pred_stream_kernel(StreamArgs a) {
 #pragma unroll
   for (int x = 0; x < 4; ++x) {                             // rows g, g + 8, g + 16, g + 24
     piv[x] = pivots[g + 8 * x];
-    zo[x] = z_off(g + 8 * x, 8 * warp + 2 * t);
+    zo[x] = z_off(g + 8 * x, 8 * (warp & 15) + 2 * t);
   }
-  const uint32_t po = kOffP + p_off(g, 8 * warp + 2 * t);           // + 1024 per output tile
+  const uint32_t po = kOffP + p_off(g, 8 * (warp & 15) + 2 * t);    // + 1024 per output tile
+  const uint32_t so0 = z_off(warp & 15, 4 * lane), so1 = z_off((warp & 15) + kWarps, 4 * lane);
+  const uint32_t ro = kOffP + p_off(pj & 31, 8 * pq);               // row sums: eight weights of output pj
 
   int st = 0;
   uint32_t parity = 0;
   bool ok = true;
-  for (int u = 0; u < n_sub; ++u) {
+  for (int u = 0; u < n_sub && warp < kWarps; ++u) {
     ok = mbar_wait(full(st), parity, s_abort);
     if (!ok) break;
     const unsigned char* zst = smem + st * kZStage;
@@ -317,21 +334,12 @@ pred_stream_kernel(StreamArgs a) {
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty(st));                  // this warp is done with the stage
-    // refill the PREVIOUS stage (one iteration late, so that nobody waits for the slowest warp)
-    if (u >= 1 && u - 1 + kStages < n_sub) {
-      const int sp = st == 0 ? kStages - 1 : st - 1;
-      const uint32_t pp = st == 0 ? parity ^ 1 : parity;    // phase of the sub-tile u - 1 in that stage
-      ok = mbar_wait(empty(sp), pp, s_abort);
-      if (!ok) break;
-      fill(u - 1 + kStages, sp);
-    }
     if (++st == kStages) { st = 0; parity ^= 1; }
   }
   __syncthreads();
   if (*s_abort) {
-    // Some wait ran out.  Let this thread's copies land before the shared memory is
-    // released, flag the status word, and leave.
-    asm volatile("cp.async.wait_all;" ::: "memory");
+    // Some wait ran out (the copy warp has already waited for its copies): flag the
+    // status word and leave.
     if (tid == 0) atomicOr(a.status, 8 /*TIMEOUT*/);
     __syncthreads();
     return;
@@ -363,19 +371,19 @@ pred_stream_kernel(StreamArgs a) {
   float* red = reinterpret_cast<float*>(smem);
   constexpr int kTile = kRowsPerCta * kPredLog;             // 1024 projections per CTA
   static_assert(kStages * kZStage >= kWarps * kTile * 4, "reduction buffer");
+  if (warp < kWarps) {
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
+    for (int h = 0; h < 2; ++h) {
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      float* q = red + warp * kTile + (16 * h + g) * kPredLog + 8 * nt + 2 * t;
-      q[0] = d[h][nt][0]; q[1] = d[h][nt][1];
-      q[8 * kPredLog] = d[h][nt][2]; q[8 * kPredLog + 1] = d[h][nt][3];
+      for (int nt = 0; nt < 4; ++nt) {
+        float* q = red + warp * kTile + (16 * h + g) * kPredLog + 8 * nt + 2 * t;
+        q[0] = d[h][nt][0]; q[1] = d[h][nt][1];
+        q[8 * kPredLog] = d[h][nt][2]; q[8 * kPredLog + 1] = d[h][nt][3];
+      }
     }
   }
   __syncthreads();
-#pragma unroll
-  for (int y = 0; y < kTile / kStreamThreads; ++y) {
-    const int e = tid + y * kStreamThreads;
+  for (int e = tid; e < kTile; e += kStreamThreads) {
     float acc = 0.f;
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) acc += red[w * kTile + e];
@@ -383,7 +391,7 @@ pred_stream_kernel(StreamArgs a) {
     if (row0 + r < live_rows)
       a.part[((size_t)(row0 + r) * a.chunks + chunk) * kPredRec + 20 + j] = acc;
   }
-  if (blockIdx.y == 0) {
+  if (blockIdx.y == 0 && warp < kWarps) {
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) p_rowsum += __shfl_xor_sync(0xffffffffu, p_rowsum, o);
     if (pq == 0) a.rowsum[chunk * kPredLog + pj] = p_rowsum;
@@ -592,6 +600,37 @@ __global__ void __launch_bounds__(256) pred_mlp_kernel(MlpArgs a) {
 
 }  // namespace
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn pred_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+// row-major [rows][inner] matrix with a row pitch, box [box_rows][box_inner], 128-byte swizzle
+static bool pred_encode(CUtensorMap* out, CUtensorMapDataType dt, const void* ptr, uint64_t inner, uint64_t rows,
+                        uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows) {
+  EncodeTiledFn enc = pred_encode_fn();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {box_inner, box_rows};
+  cuuint32_t es[2] = {1, 1};
+  return enc(out, dt, 2, const_cast<void*>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 cudaError_t predictor_prepare() {
   return cudaFuncSetAttribute(pred_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
 }
@@ -619,7 +658,18 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   StreamArgs sa{p.draft_logits, p.ld, p.vocab, p.n_live, p.n_bs,
                 reinterpret_cast<const __nv_bfloat16*>(p.p_logit), part, rowsum, chunks, chunk_len,
                 ws_ptr<int>(p.ws, L.hdr) + H_STATUS};
-  pred_stream_kernel<<<dim3(chunks, row_groups), kStreamThreads, kStreamSmem, stream>>>(sa);
+  CUtensorMap tz, tp;
+  if (!pred_encode(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, p.draft_logits, (uint64_t)p.vocab,
+                   (uint64_t)kPredPos * p.n_bs, (uint64_t)p.ld * 4, 32, kRowsPerCta))
+    return cudaErrorNotSupported;
+  if ((p.vocab & 7) == 0) {
+    if (!pred_encode(&tp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p.p_logit, (uint64_t)p.vocab, kPredLog,
+                     (uint64_t)p.vocab * 2, 64, kPredLog))
+      return cudaErrorNotSupported;
+  } else {
+    tp = tz;                                            // never used: odd vocabularies stage the matrix by hand
+  }
+  pred_stream_kernel<<<dim3(chunks, row_groups), kStreamThreads, kStreamSmem, stream>>>(sa, tz, tp);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   FeatArgs fa{p.draft_logits, p.ld, p.vocab, p.n_live, p.n_bs,
