@@ -414,7 +414,7 @@ struct FeatArgs {
   float* feat;                     // [n_bs][1735]
 };
 
-constexpr int kFeatThreads = 256;
+constexpr int kFeatThreads = 512;   // one warp per draft position
 
 __global__ void __launch_bounds__(kFeatThreads) pred_features_kernel(FeatArgs a) {
   const int i = blockIdx.x;
@@ -429,11 +429,24 @@ __global__ void __launch_bounds__(kFeatThreads) pred_features_kernel(FeatArgs a)
     for (int p = warp; p < kPredPos; p += kFeatThreads / 32) {
       const int row = i * kPredPos + p;
       const float* rec0 = a.part + (size_t)row * a.chunks * kPredRec;
-      float tv = -INFINITY, tau = -INFINITY;
-      for (int c = 0; c < a.chunks; ++c) {
-        const float cand = lane < 16 ? rec0[(size_t)c * kPredRec + lane] : -INFINITY;
-        top16_offer(tv, tau, cand, lane);
+      // all loads of this position first (independent), then the merges
+      float cand[kPredMaxChunks / 2];                       // lane l: candidate l % 16 of chunk 2 x + l / 16
+#pragma unroll
+      for (int x = 0; x < kPredMaxChunks / 2; ++x) {
+        const int c = 2 * x + (lane >> 4);
+        cand[x] = c < a.chunks ? rec0[(size_t)c * kPredRec + (lane & 15)] : -INFINITY;
       }
+      float proj = 0.f, rs = 0.f;
+#pragma unroll 8
+      for (int c = 0; c < a.chunks; ++c) {
+        proj += rec0[(size_t)c * kPredRec + 20 + lane];
+        rs += a.rowsum[c * kPredLog + lane];
+      }
+      const float pivot = a.logits[(size_t)row * a.ld];
+      float tv = -INFINITY, tau = -INFINITY;
+#pragma unroll
+      for (int x = 0; x < kPredMaxChunks / 2; ++x)
+        if (2 * x < a.chunks) top16_offer(tv, tau, cand[x], lane);
       // merge the chunks' (max, sum, sum e z, sum z): lane = chunk
       float m = -INFINITY, s_sum = 0.f, t_sum = 0.f, z_sum = 0.f;
       if (lane < a.chunks) {
@@ -460,13 +473,7 @@ __global__ void __launch_bounds__(kFeatThreads) pred_features_kernel(FeatArgs a)
       else if (lane == 16) fc[16] = top - lse;
       else if (lane == 17) fc[17] = lse - t_sum / s_sum;
       // logit projection of z - mean(z): the kernel accumulated P (z - pivot)
-      const float pivot = a.logits[(size_t)row * a.ld];
       const float mean = z_sum / (float)a.vocab;
-      float proj = 0.f, rs = 0.f;
-      for (int c = 0; c < a.chunks; ++c) {
-        proj += rec0[(size_t)c * kPredRec + 20 + lane];
-        rs += a.rowsum[c * kPredLog + lane];
-      }
       f[kPredPos * (kPredConf + kPredHid) + p * kPredLog + lane] = proj - (mean - pivot) * rs;
     }
     if (warp == 0 && lane < kPredCtx)
@@ -490,47 +497,56 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+constexpr int kHidSlices = 4;                               // grid.y: 16 of the 64 outputs each
+
 __global__ void __launch_bounds__(kHidThreads) pred_hidden_kernel(FeatArgs a) {
-  __shared__ float red[kHidThreads / 32][16 * kPredHid];
+  constexpr int kOut = kPredHid / kHidSlices;               // 16 outputs = 2 n-tiles
+  __shared__ float red[kHidThreads / 32][16 * kOut];
   int n = *a.n_live;
   n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
   const int live_rows = kPredPos * n;
   const int row0 = blockIdx.x * 16;
   if (row0 >= live_rows) return;
+  const int j0 = blockIdx.y * kOut;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int H = a.hidden_dim;
   const int r_lo = min(row0 + g, live_rows - 1), r_hi = min(row0 + g + 8, live_rows - 1);
   const __nv_bfloat16* h_lo = a.hidden + (size_t)r_lo * H;
   const __nv_bfloat16* h_hi = a.hidden + (size_t)r_hi * H;
-  float d[8][4];
+  const __nv_bfloat16* p0 = a.p_hidden + (size_t)(j0 + g) * H;
+  const __nv_bfloat16* p1 = a.p_hidden + (size_t)(j0 + 8 + g) * H;
+  float d[2][4];
 #pragma unroll
-  for (int x = 0; x < 8; ++x) d[x][0] = d[x][1] = d[x][2] = d[x][3] = 0.f;
+  for (int x = 0; x < 2; ++x) d[x][0] = d[x][1] = d[x][2] = d[x][3] = 0.f;
   const uint4 zero4 = make_uint4(0, 0, 0, 0);
-  for (int kb = warp * 32; kb < H; kb += 32 * (kHidThreads / 32)) {
+  constexpr int kStep = 32 * (kHidThreads / 32);            // columns per round of the 8 warps
+#pragma unroll 4
+  for (int kb = warp * 32; kb < H; kb += kStep) {
     const int c = kb + 8 * t;                              // hidden_dim % 8 == 0: a chunk is in or out
     const bool in = c < H;
     const uint4 alo = in ? __ldg(reinterpret_cast<const uint4*>(h_lo + c)) : zero4;
     const uint4 ahi = in ? __ldg(reinterpret_cast<const uint4*>(h_hi + c)) : zero4;
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-      const uint4 b = in ? __ldg(reinterpret_cast<const uint4*>(a.p_hidden + (size_t)(8 * nt + g) * H + c)) : zero4;
-      mma_bf16(d[nt], alo.x, ahi.x, alo.y, ahi.y, b.x, b.y);
-      mma_bf16(d[nt], alo.z, ahi.z, alo.w, ahi.w, b.z, b.w);
-    }
+    const uint4 b0 = in ? __ldg(reinterpret_cast<const uint4*>(p0 + c)) : zero4;
+    const uint4 b1 = in ? __ldg(reinterpret_cast<const uint4*>(p1 + c)) : zero4;
+    mma_bf16(d[0], alo.x, ahi.x, alo.y, ahi.y, b0.x, b0.y);
+    mma_bf16(d[0], alo.z, ahi.z, alo.w, ahi.w, b0.z, b0.w);
+    mma_bf16(d[1], alo.x, ahi.x, alo.y, ahi.y, b1.x, b1.y);
+    mma_bf16(d[1], alo.z, ahi.z, alo.w, ahi.w, b1.z, b1.w);
   }
 #pragma unroll
-  for (int nt = 0; nt < 8; ++nt) {
-    red[warp][g * kPredHid + 8 * nt + 2 * t] = d[nt][0];
-    red[warp][g * kPredHid + 8 * nt + 2 * t + 1] = d[nt][1];
-    red[warp][(g + 8) * kPredHid + 8 * nt + 2 * t] = d[nt][2];
-    red[warp][(g + 8) * kPredHid + 8 * nt + 2 * t + 1] = d[nt][3];
+  for (int nt = 0; nt < 2; ++nt) {
+    red[warp][g * kOut + 8 * nt + 2 * t] = d[nt][0];
+    red[warp][g * kOut + 8 * nt + 2 * t + 1] = d[nt][1];
+    red[warp][(g + 8) * kOut + 8 * nt + 2 * t] = d[nt][2];
+    red[warp][(g + 8) * kOut + 8 * nt + 2 * t + 1] = d[nt][3];
   }
   __syncthreads();
-  for (int x = tid; x < 16 * kPredHid; x += kHidThreads) {
+  {
+    const int x = tid;                                      // 16 rows x 16 outputs = 256 = kHidThreads
     float acc = 0.f;
 #pragma unroll
     for (int w = 0; w < kHidThreads / 32; ++w) acc += red[w][x];
-    const int row = row0 + (x >> 6), j = x & 63;
+    const int row = row0 + (x >> 4), j = j0 + (x & 15);
     if (row < live_rows) {
       const int i = row / kPredPos, p = row - i * kPredPos;
       a.feat[(size_t)i * kPredFeatures + kPredPos * kPredConf + p * kPredHid + j] = acc;
@@ -551,7 +567,9 @@ struct MlpArgs {
   float* features_out;  // nullable [n_bs][1735]
 };
 
-__global__ void __launch_bounds__(256) pred_mlp_kernel(MlpArgs a) {
+constexpr int kMlpThreads = 1024;                           // 32 warps: two hidden units each
+
+__global__ void __launch_bounds__(kMlpThreads) pred_mlp_kernel(MlpArgs a) {
   __shared__ float sf[kPredFeatures];
   __shared__ float sh[kPredMlp];
   const int i = blockIdx.x;
@@ -561,40 +579,43 @@ __global__ void __launch_bounds__(256) pred_mlp_kernel(MlpArgs a) {
   if (i >= n) {                                           // dead request: zeros
     if (tid < kPredPos) a.pred_logits[i * kPredPos + tid] = 0.f;
     if (a.features_out)
-      for (int x = tid; x < kPredFeatures; x += 256) a.features_out[(size_t)i * kPredFeatures + x] = 0.f;
+      for (int x = tid; x < kPredFeatures; x += kMlpThreads) a.features_out[(size_t)i * kPredFeatures + x] = 0.f;
     return;
   }
-  for (int x = tid; x < kPredFeatures; x += 256) {
+  for (int x = tid; x < kPredFeatures; x += kMlpThreads) {
     const float v = a.feat[(size_t)i * kPredFeatures + x];
     sf[x] = v;
     if (a.features_out) a.features_out[(size_t)i * kPredFeatures + x] = v;
   }
   __syncthreads();
   {
-    // warp w computes hidden units 8 w .. 8 w + 7 together: eight independent weight streams
-    const float* w = a.w1 + (size_t)(8 * warp) * kPredFeatures;
-    float acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    // warp w computes hidden units 2 w and 2 w + 1: many independent weight loads in flight
+    const float* w0 = a.w1 + (size_t)(2 * warp) * kPredFeatures;
+    const float* w1 = w0 + kPredFeatures;
+    float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll 8
     for (int x = lane; x < kPredFeatures; x += 32) {
       const float fx = sf[x];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[j] = fmaf(__ldg(w + (size_t)j * kPredFeatures + x), fx, acc[j]);
+      acc0 = fmaf(__ldg(w0 + x), fx, acc0);
+      acc1 = fmaf(__ldg(w1 + x), fx, acc1);
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
-      if (lane == 0) sh[8 * warp + j] = fmaxf(acc[j] + a.b1[8 * warp + j], 0.f);
+    for (int o = 16; o > 0; o >>= 1) {
+      acc0 += __shfl_xor_sync(0xffffffffu, acc0, o);
+      acc1 += __shfl_xor_sync(0xffffffffu, acc1, o);
+    }
+    if (lane == 0) {
+      sh[2 * warp] = fmaxf(acc0 + a.b1[2 * warp], 0.f);
+      sh[2 * warp + 1] = fmaxf(acc1 + a.b1[2 * warp + 1], 0.f);
     }
   }
   __syncthreads();
-  for (int o = warp; o < kPredPos; o += 8) {
-    const float* w = a.w2 + o * kPredMlp;
+  if (warp < kPredPos) {
+    const float* w = a.w2 + warp * kPredMlp;
     float acc = w[lane] * sh[lane] + w[lane + 32] * sh[lane + 32];
 #pragma unroll
     for (int x = 16; x > 0; x >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, x);
-    if (lane == 0) a.pred_logits[i * kPredPos + o] = acc + a.b2[o];
+    if (lane == 0) a.pred_logits[i * kPredPos + warp] = acc + a.b2[warp];
   }
 }
 
@@ -678,11 +699,11 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   pred_features_kernel<<<p.n_bs, kFeatThreads, 0, stream>>>(fa);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  pred_hidden_kernel<<<(kPredPos * p.n_bs + 15) / 16, kHidThreads, 0, stream>>>(fa);
+  pred_hidden_kernel<<<dim3((kPredPos * p.n_bs + 15) / 16, kHidSlices), kHidThreads, 0, stream>>>(fa);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   MlpArgs ma{p.n_live, p.n_bs, feat, p.w1, p.b1, p.w2, p.b2, p.pred_logits, p.features_out};
-  pred_mlp_kernel<<<p.n_bs, 256, 0, stream>>>(ma);
+  pred_mlp_kernel<<<p.n_bs, kMlpThreads, 0, stream>>>(ma);
   return cudaGetLastError();
 }
 
