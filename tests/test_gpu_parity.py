@@ -249,6 +249,26 @@ def test_attn_full_capacity_of_64_requests(P, impl):
     _attn_parity(P, impl, cfg, n_bs=64)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_attn_random_shapes(P, seed):
+    """Seeded sweep over live counts, capacities, head counts and context mixes (short, around
+    the 128-key tile boundary, long enough to be cut across CTAs): the tensor-core kernel against
+    the oracle, then the CUDA-core kernel against the same oracle on the same inputs."""
+    rng = np.random.default_rng(1000 + seed)
+    n_bs = int(rng.integers(1, 25))
+    n = int(rng.integers(1, n_bs + 1))
+    h_kv = int(rng.choice([1, 2, 4, 8]))
+    kinds = rng.integers(0, 4, size=n)
+    ctx = np.where(kinds == 0, rng.integers(0, 40, size=n),
+          np.where(kinds == 1, 128 * rng.integers(1, 4, size=n) + rng.integers(-2, 3, size=n),
+          np.where(kinds == 2, rng.integers(200, 1500, size=n), rng.integers(2000, 6000, size=n))))
+    if seed % 3 == 0:
+        ctx[int(rng.integers(0, n))] = int(rng.integers(12000, 30000))     # one pair over many CTAs
+    cfg = small_variant(CONFIGS["tiny"], n=n, seed=500 + seed, n_q_heads=4 * h_kv, n_kv_heads=h_kv)
+    for impl in ("tensor", "simt"):
+        _attn_parity(P, impl, cfg, n_bs=n_bs, ctx_override=[int(x) for x in ctx])
+
+
 def test_attn_simt_other_group_sizes(P):
     for hq, hkv in ((4, 4), (8, 4), (8, 1)):
         cfg = small_variant(CONFIGS["tiny"], n_q_heads=hq, n_kv_heads=hkv, seed=21)
