@@ -42,10 +42,40 @@ struct Scheduler {
   __device__ bool more() const { return pos < end; }   // runs left after the one just returned
 };
 
-__device__ __forceinline__ long long slice_begin(int c, long long T, int C) { return (long long)c * T / C; }
+// Slices are equal, except that the last two CTAs get fewer tiles.  Blocks are handed to
+// SMs in index order as the SMs fall free, so with programmatic dependent launch the
+// last block of a launch lands on the SM that finished the previous launch last: it
+// starts its preamble when the others have long finished theirs (measured: first MMA
+// 4-5 us later for the last block, 1.5 us for the one before), and with an equal share
+// it would again finish last, launch after launch.  Three tiles and one tile less
+// (about 4.8 and 1.6 us of streaming) let them finish with the rest.
+__device__ __forceinline__ void slice_skew(long long T, int C, int& d1, int& d2) {
+#ifdef DSCALE_NO_SKEW
+  const bool on = false;
+#else
+  const bool on = C >= 8 && T / C >= 24;
+#endif
+  d1 = on ? 3 : 0;
+  d2 = on ? 1 : 0;
+}
+__device__ __forceinline__ long long slice_begin(int c, long long T, int C) {
+  int d1, d2;
+  slice_skew(T, C, d1, d2);
+  const long long Tv = T + d1 + d2;                   // equal shares of a slightly longer list ...
+  if (c >= C) return T;
+  if (c == C - 1) return (long long)(C - 1) * Tv / C - d2;   // ... and the last two give some back
+  return (long long)c * Tv / C;
+}
 // the CTA whose slice holds linear tile index L
 __device__ __forceinline__ int cta_of(long long L, long long T, int C) {
-  return (int)(((L + 1) * C + T - 1) / T) - 1;
+  int d1, d2;
+  slice_skew(T, C, d1, d2);
+  if (d1) {
+    if (L >= slice_begin(C - 1, T, C)) return C - 1;
+    if (L >= slice_begin(C - 2, T, C)) return C - 2;
+  }
+  const long long Tv = T + d1 + d2;
+  return (int)(((L + 1) * C + Tv - 1) / Tv) - 1;
 }
 
 
