@@ -525,7 +525,7 @@ def main():
                          "layers); default 12 for the cpu_baseline leg, 2 per step for --impl reference")
     args = ap.parse_args()
     if args.cpu_layers <= 0:
-        args.cpu_layers = 12 if args.impl == "ours" else 2
+        args.cpu_layers = 18 if args.impl == "ours" else 2
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
