@@ -251,7 +251,8 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
  * as for dscale_accept.  One launch on `stream`, no allocation, no synchronisation;
  * the first call on a device queries the occupancy of the CTA-pair kernel and
  * should come before any stream capture.  Returns DSCALE_ERR_UNSUPPORTED for
- * hidden_dim % 64 != 0 or vocab < 16, DSCALE_ERR_WORKSPACE for an unknown ws,
+ * hidden_dim % 64 != 0 or vocab < 16 (and for more than 128 packed rows on a device
+ * that cannot keep a cluster of two CTAs resident), DSCALE_ERR_WORKSPACE for an unknown ws,
  * DSCALE_ERR_INVALID_ARG for null or misaligned pointers.
  */
 int dscale_lm_head_accept(void* ws, int n_bs, const void* hidden, const void* weight, int hidden_dim,

@@ -18,8 +18,8 @@
 //            running (max, first index); after the CTA's last tile one partial
 //            per (row, CTA) goes to the workspace.
 // More than 128 rows: pairs of CTAs (cta_group::2, further down), which halve the
-// hidden-state traffic per weight byte.  The one-CTA kernel also exists for 2-4
-// row tiles and serves when no CTA pair can be resident.
+// hidden-state traffic per weight byte.  (The one-CTA kernel is written for up to
+// four row tiles; only the one-tile form is built and used.)
 // The last CTA to finish (ticket, nobody waits) merges the partials in vocabulary
 // order -- so equal maxima resolve to the lowest index -- and runs the acceptance
 // loop of the "Prefix verifier" paragraph.
@@ -659,8 +659,7 @@ int resident_pairs(int num_ctas) {
 }  // namespace
 
 cudaError_t lm_head_prepare() {
-  const void* fns[] = {(const void*)lm_head_kernel<1>, (const void*)lm_head_kernel<2>,
-                       (const void*)lm_head_kernel<3>, (const void*)lm_head_kernel<4>,
+  const void* fns[] = {(const void*)lm_head_kernel<1>,
                        (const void*)lm_head_pair_kernel<1>, (const void*)lm_head_pair_kernel<2>};
   for (const void* f : fns) {
     cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -695,12 +694,8 @@ cudaError_t launch_lm_head(void* ws, int n_bs, const void* hidden, const void* w
       !encode_2d(&tb, weight, hidden_dim, vocab, sh.n_tile < vocab ? sh.n_tile : vocab,
                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
     return cudaErrorNotSupported;
-  switch (sh.m_tiles) {
-    case 1: lm_head_kernel<1><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb); break;
-    case 2: lm_head_kernel<2><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb); break;
-    case 3: lm_head_kernel<3><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb); break;
-    default: lm_head_kernel<4><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb); break;
-  }
+  if (sh.m_tiles != 1) return cudaErrorNotSupported;    // more than 128 rows need a resident CTA pair
+  lm_head_kernel<1><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb);
   return cudaGetLastError();
 }
 
