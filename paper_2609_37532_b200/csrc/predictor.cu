@@ -179,6 +179,37 @@ __device__ __forceinline__ void row_update(RowStat& r, float4 z, int c, int col_
   }
 }
 
+// two rows at once: the same arithmetic as row_update, written so that the two rows'
+// chains are independent instructions of one basic block
+__device__ __forceinline__ void row_update2(RowStat& a, RowStat& b, float4 za, float4 zb, int c, int col_hi,
+                                            int lane) {
+  if (c - 4 * lane + kSub > col_hi) {                       // ragged end (warp-uniform test): the careful path
+    row_update(a, za, c, col_hi, lane);
+    row_update(b, zb, c, col_hi, lane);
+    return;
+  }
+  const float la = fmaxf(fmaxf(za.x, za.y), fmaxf(za.z, za.w));
+  const float lb = fmaxf(fmaxf(zb.x, zb.y), fmaxf(zb.z, zb.w));
+  const float na = fmaxf(a.m2, la * kLog2e), nb = fmaxf(b.m2, lb * kLog2e);
+  const float fa = ex2(a.m2 - na), fb = ex2(b.m2 - nb);     // 1 when the maximum stands; m2 = -inf gives 0
+  a.s *= fa; a.t *= fa; a.m2 = na;
+  b.s *= fb; b.t *= fb; b.m2 = nb;
+  const float xa[4] = {za.x, za.y, za.z, za.w}, xb[4] = {zb.x, zb.y, zb.z, zb.w};
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {
+    const float ea = ex2(fmaf(xa[x], kLog2e, -na)), eb = ex2(fmaf(xb[x], kLog2e, -nb));
+    a.s += ea; b.s += eb;
+    a.t = fmaf(ea, xa[x], a.t); b.t = fmaf(eb, xb[x], b.t);
+    a.zsum += xa[x]; b.zsum += xb[x];
+  }
+  if (__any_sync(0xffffffffu, la > a.tau || lb > b.tau)) {  // rare once the lists have warmed up
+    top16_offer(a.tv, a.tau, za.x, lane); top16_offer(a.tv, a.tau, za.y, lane);
+    top16_offer(a.tv, a.tau, za.z, lane); top16_offer(a.tv, a.tau, za.w, lane);
+    top16_offer(b.tv, b.tau, zb.x, lane); top16_offer(b.tv, b.tau, zb.y, lane);
+    top16_offer(b.tv, b.tau, zb.z, lane); top16_offer(b.tv, b.tau, zb.w, lane);
+  }
+}
+
 __global__ void __launch_bounds__(kStreamThreads, 1)
 pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const __grid_constant__ CUtensorMap tm_p) {
   extern __shared__ unsigned char smem_raw[];
@@ -304,8 +335,10 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
     const unsigned char* pst = smem + st * kPStage;
     // ---- row statistics on the exact fp32 values
     const int c = col_lo + u * kSub + 4 * lane;
-    if (live[0]) row_update(rs[0], *reinterpret_cast<const float4*>(zst + so0), c, col_hi, lane);
-    if (live[1]) row_update(rs[1], *reinterpret_cast<const float4*>(zst + so1), c, col_hi, lane);
+    // both rows unconditionally (a dead row holds whatever the copy brought: its results are
+    // never written), so that the two dependency chains interleave
+    row_update2(rs[0], rs[1], *reinterpret_cast<const float4*>(zst + so0),
+                *reinterpret_cast<const float4*>(zst + so1), c, col_hi, lane);
     // ---- this warp's k step of the logit projection, both 16-row tiles
     {
       uint32_t bw[4];
