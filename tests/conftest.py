@@ -12,6 +12,16 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+def pytest_collection_modifyitems(config, items):
+    """Every GPU test gets a wall-clock limit (when pytest-timeout is installed): a kernel that
+    never returns must end the test, not the session."""
+    if not config.pluginmanager.hasplugin("timeout"):
+        return
+    for item in items:
+        if item.get_closest_marker("gpu") and not item.get_closest_marker("timeout"):
+            item.add_marker(pytest.mark.timeout(300))
+
+
 def read_golden(name):
     """Parse a tests/golden fixture: '#' lines are comments (the citation),
     'key: v v v' lines give integer or float lists."""
