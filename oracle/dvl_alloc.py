@@ -114,6 +114,9 @@ def dvl_alloc(n_bs: int, n_live: int, scores, draft_tokens, ctx_len, block_table
     ctx_len       [n_bs]      committed tokens already cached (anchor excluded)
     block_table   [n_bs, max_pages] physical page of logical page p
 
+    budget        total verification rows M_live (default (W/2) N, Eq. 3); any total
+                  in [N, W N] that fits the packed capacity: Eq. 9 does not depend on it
+
     Returns a dict with k, k0, offset, q_start, q_end, tokens, positions,
     kv_refs, row_req, Q, n_updates.  Packed arrays have (W/2)*n_bs slots.
     """
@@ -125,6 +128,7 @@ def dvl_alloc(n_bs: int, n_live: int, scores, draft_tokens, ctx_len, block_table
     assert 1 <= N <= n_bs
     M_bs = (W // 2) * n_bs
     M_live = (W // 2) * N if budget is None else int(budget)
+    assert N <= M_live <= min(W * N, M_bs), "budget outside [N, min(W N, capacity)]"
 
     Q = np.stack([prefix_scores(scores[i], logits_mode, W) for i in range(N)])
     k0 = [seed_length(Q[i], W) for i in range(N)]

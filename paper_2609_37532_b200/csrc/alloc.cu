@@ -90,7 +90,16 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
   // ---- 2. budget adjustment as a rank selection ----------------------------
   int sum0 = 0;
   for (int r = 0; r < N; ++r) sum0 += sK0[r];
-  const int delta = kHalfW * N - sum0;
+  // verification budget M_live: 8 N (Eq. 3) unless the caller gives one; any value in
+  // [N, 16 N] that fits the packed capacity 8 N_bs is served, others are clamped and flagged
+  int m_budget = kHalfW * N;
+  if (a.budget_rows) {
+    const int want = *a.budget_rows;
+    const int hi = min(kW * N, kHalfW * n_bs);
+    m_budget = want < N ? N : (want > hi ? hi : want);
+    if (m_budget != want && t == 0) atomicOr(&sStatus, 4 /*BAD_LEN*/);
+  }
+  const int delta = m_budget - sum0;
   if (i < N && delta != 0) {
     const int k0i = sK0[i];
     const float v = sQ[i][j];
@@ -139,7 +148,7 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
   if (t == 0) { sOff[0] = 0; sTilePre[0] = 0; }
   __syncthreads();
 
-  const int m_live = kHalfW * N;
+  const int m_live = m_budget;
   const int m_bs = kHalfW * n_bs;
   int* wk = ws_ptr<int>(a.ws, L.k);
   int* wk0 = ws_ptr<int>(a.ws, L.k0);

@@ -20,6 +20,7 @@ struct AllocArgs {
   int num_pages;
   int n_kv_heads;
   int num_ctas;
+  const int32_t* budget_rows;   // nullable device int32[1]: M_live; null = 8 N (Eq. 3)
 };
 cudaError_t launch_alloc(const AllocArgs& a, cudaStream_t stream);
 

@@ -69,6 +69,61 @@ def test_alloc_matches_oracle_random(P, seed):
     assert ws.status() == 0
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_alloc_other_budgets(P, seed):
+    """dscale_alloc_verify_budget: every total from N to min(16 N, 8 n_bs) that was sampled must
+    give the oracle's allocation bit for bit (Eq. 9 does not depend on the total)."""
+    rng = np.random.default_rng(300 + seed)
+    n_bs = int(rng.integers(2, 33))
+    n = int(rng.integers(1, n_bs + 1))
+    cfg = small_variant(CONFIGS["tiny"], n=n, seed=700 + seed)
+    req = make_requests(cfg, n_bs=n_bs)
+    hi = min(16 * n, 8 * n_bs)
+    budgets = sorted({n, n + 1, 3 * n, 8 * n - 1, 8 * n, min(8 * n + 1, hi), (n + hi) // 2, hi - 1, hi}
+                     & set(range(n, hi + 1)))
+    ws = _ws(P, req)
+    st = StagedRequests(req)
+    for b in budgets:
+        got = gpu_alloc(P, ws, st, budget=b)
+        assert_alloc_equal(got, oracle_alloc(req, budget=b))
+        assert int(got["k"][:n].sum()) == b and int(got["offset"][n]) == b
+    assert ws.status() == 0
+    # out of range: clamped and flagged
+    got = gpu_alloc(P, ws, st, budget=n - 1)
+    assert_alloc_equal(got, oracle_alloc(req, budget=n))
+    assert ws.status() & 4
+    ws2 = _ws(P, req)
+    got = gpu_alloc(P, ws2, st, budget=16 * n_bs + 5)
+    assert_alloc_equal(got, oracle_alloc(req, budget=hi))
+    assert ws2.status() & 4
+
+
+def test_other_budget_through_attention_and_accept(P):
+    """A step under a budget of 13 rows per request: the downstream calls read M_live from the
+    workspace and need no other change."""
+    cfg = small_variant(CONFIGS["tiny"], n=4, seed=77, vocab=2048)
+    req, _, kc, vc, qu, _ = full_case(cfg, n_bs=8)
+    n, n_bs, b = 4, 8, 52
+    alloc = oracle_alloc(req, budget=b)
+    ws = _ws(P, req)
+    st = StagedRequests(req)
+    assert_alloc_equal(gpu_alloc(P, ws, st, budget=b), alloc)
+    qp = rows_to_packed(qu, alloc["k"], alloc["offset"], n, 8 * n_bs)
+    out = torch.full(qp.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    P.verify_attn(ws, qp.cuda(), kc.cuda(), vc.cuda(), st.block_table, SCALE, out)
+    torch.cuda.synchronize()
+    ok, max_abs, worst = attn_close(out, oracle_attn(req, alloc, kc, vc, qp))
+    assert ok, (max_abs, worst)
+    assert (out[b:].float() == 0).all()
+    lp = rows_to_packed(make_logits_unpacked(req), alloc["k"], alloc["offset"], n, 8 * n_bs)
+    got = gpu_accept(P, ws, lp.cuda(), cfg.vocab, n_bs)
+    exp = oracle_accept(req, alloc, lp)
+    np.testing.assert_array_equal(got["top1"][:b], exp["top1"][:b])
+    for f in ("accept_len", "next_anchor", "out_tokens", "out_len"):
+        np.testing.assert_array_equal(got[f], exp[f], err_msg=f)
+    assert ws.status() == 0
+
+
 def test_alloc_extremes(P):
     cfg = small_variant(CONFIGS["tiny"], n=64, seed=9)
     for fill in (0.0, 1.0, 0.5):

@@ -177,6 +177,28 @@ def _brute_best(Q, k0, budget, W, grow):
 
 
 @pytest.mark.parametrize("seed", range(10))
+def test_prop1_bruteforce_other_budgets(seed):
+    """Eq. 9 for totals other than (W/2) N: the greedy result is optimal among all allocations
+    reachable by only growing (or only shrinking) the seeds, for every budget in [N, W N]."""
+    rng = np.random.default_rng(900 + seed)
+    W, n = 5, 4
+    s = np.sort(rng.uniform(0, 1, size=(n, W - 1)), axis=1)[:, ::-1].astype(np.float32)
+    if seed % 2 == 0:
+        s = np.round(s * 4) / 4
+    Q = np.stack([O.prefix_scores(s[i], W=W) for i in range(n)])
+    k0 = [O.seed_length(Q[i], W=W) for i in range(n)]
+    for budget in range(n, W * n + 1):
+        k, upd = O.budget_adjust(Q, k0, budget, W=W)
+        assert sum(k) == budget and upd == abs(budget - sum(k0)) and all(1 <= x <= W for x in k)
+        d0 = budget - sum(k0)
+        if d0 == 0:
+            assert k == k0
+        else:
+            best = _brute_best(Q, k0, budget, W, grow=d0 > 0)
+            assert abs(O.prefix_objective(Q, k) - best) < 1e-9
+
+
+@pytest.mark.parametrize("seed", range(10))
 def test_prop1_bruteforce_small_W(seed):
     rng = np.random.default_rng(100 + seed)
     W, n = 6, 4
