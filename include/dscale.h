@@ -131,18 +131,23 @@ int dscale_alloc_verify(void* ws, int n_bs, const int32_t* n_live, const float* 
                         int num_pages, void* stream);
 
 /*
- * The same allocation under another verification budget (the budget of Eq. 3 is
- * M_live = W N / 2 = 8 N; Section 3.3's allocator and Eq. 9 hold for any total).
- * budget_rows is a device int32[1] read by the kernel: sum_i k_i = budget_rows.
- * Served range: N <= budget_rows <= min(16 N, 8 n_bs) (every request keeps its
- * anchor, no request exceeds its 16 slots, the packed arrays keep their 8 n_bs
+ * The same allocation for another block width and / or another verification
+ * budget.  block_width = W is the number of slots a request's block has (even,
+ * 2..16; the paper's drafters have 16 and it leaves other widths open): only the
+ * first W - 1 scores and W draft tokens of each row are read (the array shapes
+ * stay [n_bs][15] and [n_bs][16]), seeds are clipped to [1, W], no request grows
+ * beyond W.  budget_rows is a nullable device int32[1] read by the kernel:
+ * sum_i k_i = budget_rows; null means W N / 2 (Eq. 3; Eq. 9 holds for any
+ * total).  Served range: N <= budget_rows <= min(W N, 8 n_bs) (every request
+ * keeps its anchor, none exceeds its block, the packed arrays keep their 8 n_bs
  * rows); a value outside is clamped into the range and DSCALE_STATUS_BAD_LEN is
- * set.  Everything downstream reads M_live from the workspace and needs no change.
+ * set.  Everything downstream reads M_live from the workspace and needs no
+ * change.  DSCALE_ERR_UNSUPPORTED for an odd or out-of-range block_width.
  */
-int dscale_alloc_verify_budget(void* ws, int n_bs, const int32_t* n_live, const float* scores,
-                               int scores_are_logits, const int32_t* draft_tokens,
-                               const int32_t* ctx_len, const int32_t* block_table, int max_pages,
-                               int num_pages, const int32_t* budget_rows, void* stream);
+int dscale_alloc_verify_ex(void* ws, int n_bs, const int32_t* n_live, const float* scores,
+                           int scores_are_logits, const int32_t* draft_tokens,
+                           const int32_t* ctx_len, const int32_t* block_table, int max_pages,
+                           int num_pages, int block_width, const int32_t* budget_rows, void* stream);
 
 /*
  * Packed ragged verify attention for one layer (Section 3.2; Eq. 15 and the

@@ -106,7 +106,8 @@ def offsets_of(k) -> list:
 
 
 def dvl_alloc(n_bs: int, n_live: int, scores, draft_tokens, ctx_len, block_table,
-              logits_mode: bool = False, W: int = W_DEFAULT, budget: int | None = None):
+              logits_mode: bool = False, W: int = W_DEFAULT, budget: int | None = None,
+              capacity: int | None = None):
     """Whole of Algorithm 1 from the scores down.
 
     scores        [n_bs, W-1] float32, slot j=1..W-1
@@ -116,6 +117,7 @@ def dvl_alloc(n_bs: int, n_live: int, scores, draft_tokens, ctx_len, block_table
 
     budget        total verification rows M_live (default (W/2) N, Eq. 3); any total
                   in [N, W N] that fits the packed capacity: Eq. 9 does not depend on it
+    capacity      rows of the packed arrays (default (W/2) n_bs, the paper's M_bs)
 
     Returns a dict with k, k0, offset, q_start, q_end, tokens, positions,
     kv_refs, row_req, Q, n_updates.  Packed arrays have (W/2)*n_bs slots.
@@ -126,7 +128,7 @@ def dvl_alloc(n_bs: int, n_live: int, scores, draft_tokens, ctx_len, block_table
     block_table = np.asarray(block_table)
     N = int(n_live)
     assert 1 <= N <= n_bs
-    M_bs = (W // 2) * n_bs
+    M_bs = (W // 2) * n_bs if capacity is None else int(capacity)
     M_live = (W // 2) * N if budget is None else int(budget)
     assert N <= M_live <= min(W * N, M_bs), "budget outside [N, min(W N, capacity)]"
 

@@ -25,8 +25,8 @@ lib.dscale_workspace_init.restype = _i
 lib.dscale_workspace_init.argtypes = [_vp, _sz, _i, _i, _i, _i, _i, _vp]
 lib.dscale_alloc_verify.restype = _i
 lib.dscale_alloc_verify.argtypes = [_vp, _i, _vp, _vp, _i, _vp, _vp, _vp, _i, _i, _vp]
-lib.dscale_alloc_verify_budget.restype = _i
-lib.dscale_alloc_verify_budget.argtypes = [_vp, _i, _vp, _vp, _i, _vp, _vp, _vp, _i, _i, _vp, _vp]
+lib.dscale_alloc_verify_ex.restype = _i
+lib.dscale_alloc_verify_ex.argtypes = [_vp, _i, _vp, _vp, _i, _vp, _vp, _vp, _i, _i, _i, _vp, _vp]
 for _name in ("dscale_verify_attn", "dscale_verify_attn_simt"):
     getattr(lib, _name).restype = _i
     getattr(lib, _name).argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _f, _vp, _vp]
@@ -126,20 +126,22 @@ class VerifyWorkspace:
 
 
 def alloc_verify(ws: VerifyWorkspace, n_live, scores, draft_tokens, ctx_len, block_table,
-                 num_pages: int, scores_are_logits: bool = False, budget_rows=None):
-    """DVL allocation; budget_rows (device int32[1]) selects dscale_alloc_verify_budget."""
+                 num_pages: int, scores_are_logits: bool = False, budget_rows=None, block_width: int = 16):
+    """DVL allocation; a budget_rows tensor (device int32[1]) or a block width other than 16
+    goes through dscale_alloc_verify_ex."""
     _need(n_live, torch.int32, "n_live"); _need(scores, torch.float32, "scores")
     _need(draft_tokens, torch.int32, "draft_tokens"); _need(ctx_len, torch.int32, "ctx_len")
     _need(block_table, torch.int32, "block_table")
     assert scores.shape == (ws.n_bs, 15) and draft_tokens.shape == (ws.n_bs, 16)
     assert ctx_len.shape == (ws.n_bs,) and block_table.shape[0] == ws.n_bs
-    if budget_rows is not None:
-        _need(budget_rows, torch.int32, "budget_rows")
-        _check(lib.dscale_alloc_verify_budget(C.c_void_p(ws.ptr), ws.n_bs, _ptr(n_live), _ptr(scores),
-                                              int(scores_are_logits), _ptr(draft_tokens), _ptr(ctx_len),
-                                              _ptr(block_table), block_table.shape[1], num_pages,
-                                              _ptr(budget_rows), _stream()),
-               "dscale_alloc_verify_budget")
+    if budget_rows is not None or block_width != 16:
+        if budget_rows is not None:
+            _need(budget_rows, torch.int32, "budget_rows")
+        _check(lib.dscale_alloc_verify_ex(C.c_void_p(ws.ptr), ws.n_bs, _ptr(n_live), _ptr(scores),
+                                          int(scores_are_logits), _ptr(draft_tokens), _ptr(ctx_len),
+                                          _ptr(block_table), block_table.shape[1], num_pages, int(block_width),
+                                          _ptr(budget_rows), _stream()),
+               "dscale_alloc_verify_ex")
         return
     _check(lib.dscale_alloc_verify(C.c_void_p(ws.ptr), ws.n_bs, _ptr(n_live), _ptr(scores),
                                    int(scores_are_logits), _ptr(draft_tokens), _ptr(ctx_len),

@@ -51,6 +51,7 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
   const int t = threadIdx.x;
   const int i = t >> 4, j = t & 15;
   const int n_bs = a.n_bs;
+  const int Wd = a.block_width;                       // slots per request that exist (<= kW)
   int* hdr = ws_ptr<int>(a.ws, L.hdr);
 
   if (t == 0) sStatus = 0;
@@ -68,7 +69,8 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
     int st = 0;
     float q = 1.0f, lhat = 0.0f;
     sQ[i][0] = 1.0f;
-    for (int jj = 1; jj < kW; ++jj) {
+    for (int jj = Wd; jj < kW; ++jj) sQ[i][jj] = 0.0f;    // slots a narrower block does not have
+    for (int jj = 1; jj < Wd; ++jj) {
       float s = a.scores[i * (kW - 1) + jj - 1];
       if (a.scores_are_logits) s = (float)(1.0 / (1.0 + exp(-(double)s)));
       if (!(s >= 0.0f)) { s = 0.0f; st |= 1; }      // NaN or negative
@@ -78,7 +80,7 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
       lhat = __fadd_rn(lhat, q);                    // Eq. 7, left to right
     }
     int r = (int)floorf(__fadd_rn(lhat, 0.5f));
-    sK0[i] = min(kW, max(1, r));
+    sK0[i] = min(Wd, max(1, r));
     int c = a.ctx_len[i];
     const int c_max = a.max_pages * kPage - kW;
     if (c < 0 || c > c_max) { st |= 4; c = c < 0 ? 0 : c_max; }
@@ -92,10 +94,10 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
   for (int r = 0; r < N; ++r) sum0 += sK0[r];
   // verification budget M_live: 8 N (Eq. 3) unless the caller gives one; any value in
   // [N, 16 N] that fits the packed capacity 8 N_bs is served, others are clamped and flagged
-  int m_budget = kHalfW * N;
+  int m_budget = (Wd / 2) * N;
   if (a.budget_rows) {
     const int want = *a.budget_rows;
-    const int hi = min(kW * N, kHalfW * n_bs);
+    const int hi = min(Wd * N, kHalfW * n_bs);
     m_budget = want < N ? N : (want > hi ? hi : want);
     if (m_budget != want && t == 0) atomicOr(&sStatus, 4 /*BAD_LEN*/);
   }
@@ -103,14 +105,14 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
   if (i < N && delta != 0) {
     const int k0i = sK0[i];
     const float v = sQ[i][j];
-    if (delta > 0 && j >= k0i) {
+    if (delta > 0 && j >= k0i && j < Wd) {
       int rank = j - k0i;
       for (int r = 0; r < N && rank < delta; ++r) {
         if (r == i) continue;
         const int k0r = sK0[r];
         int c = 0;
-        if (r < i) { for (int jj = k0r; jj < kW && sQ[r][jj] >= v; ++jj) ++c; }
-        else       { for (int jj = k0r; jj < kW && sQ[r][jj] >  v; ++jj) ++c; }
+        if (r < i) { for (int jj = k0r; jj < Wd && sQ[r][jj] >= v; ++jj) ++c; }
+        else       { for (int jj = k0r; jj < Wd && sQ[r][jj] >  v; ++jj) ++c; }
         rank += c;
       }
       if (rank < delta) atomicAdd(&sAdj[i], 1);

@@ -77,7 +77,8 @@ int dscale_workspace_init(void* ws, size_t bytes, int n_bs, int n_q_heads, int n
 static int alloc_common(void* ws, int n_bs, const int32_t* n_live, const float* scores,
                         int scores_are_logits, const int32_t* draft_tokens, const int32_t* ctx_len,
                         const int32_t* block_table, int max_pages, int num_pages,
-                        const int32_t* budget_rows, void* stream) {
+                        const int32_t* budget_rows, int block_width, void* stream) {
+  if (block_width < 2 || block_width > DSCALE_W || (block_width & 1)) return DSCALE_ERR_UNSUPPORTED;
   if (!ws || !n_live || !scores || !draft_tokens || !ctx_len || !block_table)
     return DSCALE_ERR_INVALID_ARG;
   if (max_pages < 1 || num_pages < 1) return DSCALE_ERR_INVALID_ARG;
@@ -87,7 +88,7 @@ static int alloc_common(void* ws, int n_bs, const int32_t* n_live, const float* 
   WsInfo info;
   if (!lookup(ws, n_bs, &info)) return DSCALE_ERR_WORKSPACE;
   AllocArgs a{ws, n_bs, n_live, scores, scores_are_logits ? 1 : 0, draft_tokens, ctx_len,
-              block_table, max_pages, num_pages, info.n_kv_heads, info.num_ctas, budget_rows};
+              block_table, max_pages, num_pages, info.n_kv_heads, info.num_ctas, budget_rows, block_width};
   return launch_alloc(a, (cudaStream_t)stream) == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
 }
 
@@ -96,16 +97,15 @@ int dscale_alloc_verify(void* ws, int n_bs, const int32_t* n_live, const float* 
                         const int32_t* ctx_len, const int32_t* block_table, int max_pages,
                         int num_pages, void* stream) {
   return alloc_common(ws, n_bs, n_live, scores, scores_are_logits, draft_tokens, ctx_len, block_table,
-                      max_pages, num_pages, nullptr, stream);
+                      max_pages, num_pages, nullptr, DSCALE_W, stream);
 }
 
-int dscale_alloc_verify_budget(void* ws, int n_bs, const int32_t* n_live, const float* scores,
-                               int scores_are_logits, const int32_t* draft_tokens,
-                               const int32_t* ctx_len, const int32_t* block_table, int max_pages,
-                               int num_pages, const int32_t* budget_rows, void* stream) {
-  if (!budget_rows) return DSCALE_ERR_INVALID_ARG;
+int dscale_alloc_verify_ex(void* ws, int n_bs, const int32_t* n_live, const float* scores,
+                           int scores_are_logits, const int32_t* draft_tokens,
+                           const int32_t* ctx_len, const int32_t* block_table, int max_pages,
+                           int num_pages, int block_width, const int32_t* budget_rows, void* stream) {
   return alloc_common(ws, n_bs, n_live, scores, scores_are_logits, draft_tokens, ctx_len, block_table,
-                      max_pages, num_pages, budget_rows, stream);
+                      max_pages, num_pages, budget_rows, block_width, stream);
 }
 
 static int attn_common(void* ws, int n_bs, const void* q, const void* k_cache, const void* v_cache,

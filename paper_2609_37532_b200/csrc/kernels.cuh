@@ -20,7 +20,8 @@ struct AllocArgs {
   int num_pages;
   int n_kv_heads;
   int num_ctas;
-  const int32_t* budget_rows;   // nullable device int32[1]: M_live; null = 8 N (Eq. 3)
+  const int32_t* budget_rows;   // nullable device int32[1]: M_live; null = (W / 2) N (Eq. 3)
+  int block_width;              // W: slots per request that exist (even, 2..16)
 };
 cudaError_t launch_alloc(const AllocArgs& a, cudaStream_t stream);
 

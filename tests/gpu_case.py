@@ -44,15 +44,17 @@ class StagedRequests:
         self.block_table.copy_(torch.as_tensor(req["block_table"]))
 
 
-def oracle_alloc(req, logits_mode=False, budget=None):
-    return OA.dvl_alloc(req["n_bs"], req["n_live"], req["scores"], req["draft_tokens"],
-                        req["ctx_len"], req["block_table"], logits_mode=logits_mode, budget=budget)
+def oracle_alloc(req, logits_mode=False, budget=None, block_width=16):
+    W = block_width
+    return OA.dvl_alloc(req["n_bs"], req["n_live"], req["scores"][:, : W - 1], req["draft_tokens"][:, :W],
+                        req["ctx_len"], req["block_table"], logits_mode=logits_mode, W=W, budget=budget,
+                        capacity=8 * req["n_bs"])
 
 
-def gpu_alloc(P, ws, st: StagedRequests, logits_mode=False, budget=None):
+def gpu_alloc(P, ws, st: StagedRequests, logits_mode=False, budget=None, block_width=16):
     b = None if budget is None else torch.tensor([budget], dtype=torch.int32, device="cuda")
     P.alloc_verify(ws, st.n_live, st.scores, st.draft, st.ctx_len, st.block_table,
-                   st.req["num_pages"], scores_are_logits=logits_mode, budget_rows=b)
+                   st.req["num_pages"], scores_are_logits=logits_mode, budget_rows=b, block_width=block_width)
     torch.cuda.synchronize()
     return {f: ws.field(f).cpu().numpy().copy() for f in ALLOC_FIELDS}
 

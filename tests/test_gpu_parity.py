@@ -98,6 +98,35 @@ def test_alloc_other_budgets(P, seed):
     assert ws2.status() & 4
 
 
+@pytest.mark.parametrize("W", [2, 4, 8, 12])
+def test_alloc_other_block_widths(P, W):
+    """dscale_alloc_verify_ex with a narrower block: the oracle run with the same W on the first
+    W - 1 scores and W tokens.  The workspace keeps its 8 n_bs packed rows, the oracle's arrays have
+    (W / 2) n_bs: the common prefix must agree bit for bit, default and other budgets."""
+    for seed in range(3):
+        rng = np.random.default_rng(40 * W + seed)
+        n_bs = int(rng.integers(2, 40))
+        n = int(rng.integers(1, n_bs + 1))
+        cfg = small_variant(CONFIGS["tiny"], n=n, seed=800 + 10 * W + seed)
+        req = make_requests(cfg, n_bs=n_bs)
+        ws = _ws(P, req)
+        st = StagedRequests(req)
+        hi = min(W * n, 8 * n_bs)
+        for budget in (None, n, hi, (n + hi) // 2):
+            got = gpu_alloc(P, ws, st, budget=budget, block_width=W)
+            exp = oracle_alloc(req, budget=budget, block_width=W)
+            for f in ALLOC_FIELDS:
+                m = len(exp[f])
+                np.testing.assert_array_equal(got[f][:m], exp[f], err_msg=f"W={W} budget={budget} field {f}")
+            assert got["k"][:n].max() <= W and got["k"][:n].min() >= 1
+        assert ws.status() == 0
+    import ctypes as C
+    assert P.lib.dscale_alloc_verify_ex(C.c_void_p(ws.ptr), n_bs, None, None, 0, None, None, None, 1, 1, 7,
+                                        None, None) == -2          # odd width
+    assert P.lib.dscale_alloc_verify_ex(C.c_void_p(ws.ptr), n_bs, None, None, 0, None, None, None, 1, 1, 18,
+                                        None, None) == -2          # wider than the 16 slots there are
+
+
 def test_other_budget_through_attention_and_accept(P):
     """A step under a budget of 13 rows per request: the downstream calls read M_live from the
     workspace and need no other change."""
