@@ -127,16 +127,18 @@ def test_alloc_other_block_widths(P, W):
                                         None, None) == -2          # wider than the 16 slots there are
 
 
-def test_other_budget_through_attention_and_accept(P):
-    """A step under a budget of 13 rows per request: the downstream calls read M_live from the
-    workspace and need no other change."""
+@pytest.mark.parametrize("W,budget", [(16, 52), (8, None), (8, 29), (4, None)])
+def test_other_budget_and_width_through_attention_and_accept(P, W, budget):
+    """A step under another budget (13 rows per request) or a narrower block: the downstream calls
+    read M_live, lengths and offsets from the workspace and need no other change."""
     cfg = small_variant(CONFIGS["tiny"], n=4, seed=77, vocab=2048)
     req, _, kc, vc, qu, _ = full_case(cfg, n_bs=8)
-    n, n_bs, b = 4, 8, 52
-    alloc = oracle_alloc(req, budget=b)
+    n, n_bs = 4, 8
+    b = (W // 2) * n if budget is None else budget
+    alloc = oracle_alloc(req, budget=budget, block_width=W)
     ws = _ws(P, req)
     st = StagedRequests(req)
-    assert_alloc_equal(gpu_alloc(P, ws, st, budget=b), alloc)
+    assert_alloc_equal(gpu_alloc(P, ws, st, budget=budget, block_width=W), alloc)
     qp = rows_to_packed(qu, alloc["k"], alloc["offset"], n, 8 * n_bs)
     out = torch.full(qp.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
     P.verify_attn(ws, qp.cuda(), kc.cuda(), vc.cuda(), st.block_table, SCALE, out)
