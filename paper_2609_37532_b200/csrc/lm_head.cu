@@ -121,7 +121,7 @@ __device__ __forceinline__ void scan_acc(uint32_t taddr, int n, int col0, int vo
 __device__ __forceinline__ void lm_finish(const LmArgs& a, const WsLayout& L, int* hdr, int m_live,
                                           const float* best, const int* best_i, const int* rows, int n_m,
                                           int part, int n_parts, int n_ctas, bool ok, uint32_t bar_group,
-                                          volatile int* s_abort, int* s_last, int tid) {
+                                          volatile int* s_abort, int* s_last, int tid, int* scratch) {
   float* pv = ws_ptr<float>(a.ws, L.lm_val);
   int* pi = ws_ptr<int>(a.ws, L.lm_idx);
 #pragma unroll
@@ -147,6 +147,9 @@ __device__ __forceinline__ void lm_finish(const LmArgs& a, const WsLayout& L, in
   if (tid == 0) hdr[H_LM_TICKET] = 0;                 // ready for the next launch
   int* top1 = ws_ptr<int>(a.ws, L.top1);
   const int m_bs = kHalfW * a.n_bs;
+  const int* wtok = ws_ptr<int>(a.ws, L.tokens);
+  int* s_top1 = scratch;                              // the operand ring is idle by now
+  int* s_tok = scratch + m_bs;
   for (int r = tid; r < m_bs; r += kEpiThreads) {
     int bi = 0;
     if (r < m_live) {
@@ -161,21 +164,23 @@ __device__ __forceinline__ void lm_finish(const LmArgs& a, const WsLayout& L, in
       if (a.row_max) a.row_max[r] = bv;
     }
     top1[r] = bi;
+    s_top1[r] = bi;
+    s_tok[r] = wtok[r];
   }
   ok = group_sync();
   const int N = hdr[H_N_LIVE];
   const int* wk = ws_ptr<int>(a.ws, L.k);
   const int* woff = ws_ptr<int>(a.ws, L.offset);
-  const int* wtok = ws_ptr<int>(a.ws, L.tokens);
   if (ok && tid < a.n_bs) {
     const int i = tid;
     int32_t* ot = a.out_tokens + i * kW;
     if (i < N) {
+      // a chain of dependent reads: on the shared-memory copies, not on global memory
       const int ki = wk[i], oi = woff[i];
       int acc = 0;
-      while (acc < ki - 1 && top1[oi + acc] == wtok[oi + acc + 1]) ++acc;
-      const int nxt = top1[oi + acc];
-      for (int j = 0; j < kW; ++j) ot[j] = j < acc ? wtok[oi + 1 + j] : (j == acc ? nxt : -1);
+      while (acc < ki - 1 && s_top1[oi + acc] == s_tok[oi + acc + 1]) ++acc;
+      const int nxt = s_top1[oi + acc];
+      for (int j = 0; j < kW; ++j) ot[j] = j < acc ? s_tok[oi + 1 + j] : (j == acc ? nxt : -1);
       a.accept_len[i] = acc;
       a.next_anchor[i] = nxt;
       a.out_len[i] = acc + 1;
@@ -321,7 +326,8 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
       tc_fence_before();
       mbar_arrive(bar(B_ACC_EMPTY));
     }
-    lm_finish(a, L, hdr, m_live, best, best_i, rows, M_TILES, c, C, C, ok, bar(B_GROUP), s_abort, s_last, tid);
+    lm_finish(a, L, hdr, m_live, best, best_i, rows, M_TILES, c, C, C, ok, bar(B_GROUP), s_abort, s_last, tid,
+              reinterpret_cast<int*>(sm));
   }
 
   tc_fence_before();
@@ -551,7 +557,7 @@ lm_head_pair_kernel(LmArgs a, WsLayout L, PairShape sh, const __grid_constant__ 
       mbar_arrive_cluster(acc_empty);
     }
     lm_finish(a, L, hdr, m_live, best, best_i, rows, M_PAIRS, pair, n_pairs, (int)gridDim.x, ok,
-              bar(B_GROUP), s_abort, s_last, tid);
+              bar(B_GROUP), s_abort, s_last, tid, reinterpret_cast<int*>(sm));
   }
 
   tc_fence_before();
