@@ -330,7 +330,10 @@ def run_ours(args, rank, world, local_rank):
             g_attn.replay()
             ev[s][1].record(stream)
         barrier()
-        attn_ms = float(np.mean([a.elapsed_time(b) for a, b in ev])) / max(1, cfg.layers)
+        _per = np.array([a.elapsed_time(b) for a, b in ev]) / max(1, cfg.layers)
+        if os.environ.get("DSCALE_BENCH_DEBUG"):
+            print("attn per-launch us by replay:", np.round(_per * 1e3, 1).tolist(), file=sys.stderr)
+        attn_ms = float(np.mean(_per))
         ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ea.record(stream)
         for _ in range(args.steps):

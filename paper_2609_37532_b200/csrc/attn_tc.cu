@@ -343,7 +343,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           const int b = pt & 1;
           const unsigned uv = 2 * pt + 1;
           const int slot = uv % kStages;
-          if (mbar_try(bar(B_P_FULL + b), (pt >> 1) & 1) && mbar_try(bar(B_KV_FULL + slot), (uv / kStages) & 1)) {
+          if (mbar_test(bar(B_P_FULL + b), (pt >> 1) & 1) && mbar_test(bar(B_KV_FULL + slot), (uv / kStages) & 1)) {
             tc_fence_after();
             const uint32_t p_base = base + kOffP + b * kPBytes;
             const uint32_t v_base = base + kOffKV + slot * kSlotBytes;
@@ -369,10 +369,10 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
             ++seg; t = sg.t0; t_end = sg.t1; q_ready = false;
           }
           const int qb = seg & 1;
-          if (!q_ready) q_ready = mbar_try(bar(B_Q_FULL + qb), (seg >> 1) & 1);
+          if (!q_ready) q_ready = mbar_test(bar(B_Q_FULL + qb), (seg >> 1) & 1);
           const unsigned uk = 2 * next_s;
           const int slot = uk % kStages;
-          if (q_ready && mbar_try(bar(B_KV_FULL + slot), (uk / kStages) & 1)) {
+          if (q_ready && mbar_test(bar(B_KV_FULL + slot), (uk / kStages) & 1)) {
             tc_fence_after();
             const int b3 = next_s % 3;
             const uint32_t q_base = base + kOffQ + qb * kQBytes;
