@@ -418,12 +418,12 @@ def run_ours(args, rank, world, local_rank):
         hs.h_ctx_len.copy_(torch.as_tensor(req["ctx_len"]))
         hs.h_block_table.copy_(torch.as_tensor(req["block_table"]))
         for _ in range(max(1, args.warmup)):
-            hs.run(); stream.synchronize()
+            hs.run(graph=True); stream.synchronize()
         barrier()
         t0 = time.perf_counter()
         e2e_tokens = 0
         for _ in range(args.steps):
-            hs.run()
+            hs.run(graph=True)
             stream.synchronize()                      # the caller reads the outputs every step
             e2e_tokens += int(hs.h_out_len.sum())
         e2e_s = time.perf_counter() - t0
@@ -465,7 +465,7 @@ def run_ours(args, rank, world, local_rank):
             "lm_head_accept": lm, "predict_scores": pred,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": hs.h2d_bytes,
                     "d2h_bytes_per_step": hs.d2h_bytes, "ms_per_step": 1e3 * e2e_s / args.steps,
-                    "api": "dscale_verify_step_host (pinned host inputs/outputs, KV/Q/logits resident)"},
+                    "api": "dscale_verify_step_host_graph (pinned host inputs/outputs, KV/Q/logits resident)"},
             "gpu_launches": args.steps * (P.lib.dscale_launches_per_call(0) +
                                           cfg.layers * P.lib.dscale_launches_per_call(1 if args.attn == "tensor" else 3) +
                                           P.lib.dscale_launches_per_call(2)),

@@ -252,6 +252,26 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
                             int32_t* h_out_tokens, int32_t* h_out_len, void* stream);
 
 /*
+ * The same step as ONE replayed CUDA graph, which is what Algorithm 2 does: stage
+ * the inputs at fixed addresses, replay, read the outputs (lines 10-21).  Same
+ * arguments and results as dscale_verify_step_host.  The first call with a given
+ * set of arguments captures the copies and launches into a graph and instantiates
+ * it (this allocates driver memory and takes about a millisecond); later calls
+ * with the same pointers and sizes only launch that graph.  One graph is kept per
+ * workspace; other arguments replace it.  The host buffers must stay where they
+ * are between calls (their addresses are part of the graph) and must be
+ * page-locked.  If `stream` is already being captured, or is the legacy default
+ * stream, the call degrades to dscale_verify_step_host.
+ */
+int dscale_verify_step_host_graph(void* ws, int n_bs, const int32_t* h_n_live, const float* h_scores,
+                                  const int32_t* h_draft_tokens, const int32_t* h_ctx_len,
+                                  const int32_t* h_block_table, int max_pages, int num_pages,
+                                  void* staging, const dscale_layer* layers, int n_layers,
+                                  int n_q_heads, int n_kv_heads, float sm_scale, const float* logits,
+                                  int64_t ld, int vocab, int32_t* h_accept_len, int32_t* h_next_anchor,
+                                  int32_t* h_out_tokens, int32_t* h_out_len, void* stream);
+
+/*
  * Fused LM head + greedy prefix verification: dscale_accept without the logits.
  * The target token of packed row s is argmax_v sum_h hidden[s][h] * weight[v][h]
  * (the LM head applied to the M = 8N packed rows DVL leaves: Section 2.2 and the

@@ -44,6 +44,8 @@ lib.dscale_verify_step_host.restype = _i
 lib.dscale_verify_step_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _i, _vp,
                                         C.POINTER(LayerPtrs), _i, _i, _i, _f, _vp, _i64, _i,
                                         _vp, _vp, _vp, _vp, _vp]
+lib.dscale_verify_step_host_graph.restype = _i
+lib.dscale_verify_step_host_graph.argtypes = lib.dscale_verify_step_host.argtypes
 lib.dscale_verify_attn_padded.restype = _i
 lib.dscale_verify_attn_padded.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i, _i, _vp, _i, _i, _f, _vp, _vp]
 lib.dscale_accept_static.restype = _i
@@ -216,9 +218,11 @@ class HostStep:
         self.h2d_bytes = 4 + n_bs * (15 + 16 + 1 + max_pages) * 4
         self.d2h_bytes = n_bs * (1 + 1 + 16 + 1) * 4
 
-    def run(self):
+    def run(self, graph: bool = False):
+        """Enqueue one step; graph=True goes through dscale_verify_step_host_graph."""
         ws = self.ws
-        _check(lib.dscale_verify_step_host(
+        fn = lib.dscale_verify_step_host_graph if graph else lib.dscale_verify_step_host
+        _check(fn(
             C.c_void_p(ws.ptr), ws.n_bs, _ptr(self.h_n_live), _ptr(self.h_scores),
             _ptr(self.h_draft), _ptr(self.h_ctx_len), _ptr(self.h_block_table), self.max_pages,
             self.num_pages, C.c_void_p(self.staging_ptr), self.table, len(self.table),

@@ -2,8 +2,10 @@
 // and dispatch to the kernel launchers.  No computation happens here.
 #include <cuda_runtime.h>
 
+#include <cstring>
 #include <map>
 #include <mutex>
+#include <vector>
 
 #include "../../include/dscale.h"
 #include "kernels.cuh"
@@ -257,6 +259,71 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
       !d2h(h_out_len, S.out_len, size_t(n_bs) * 4))
     return DSCALE_ERR_CUDA;
   return DSCALE_OK;
+}
+
+namespace {
+// one instantiated graph of the host-driven step per workspace, keyed by every argument
+struct StepGraph {
+  std::vector<uintptr_t> key;
+  cudaGraphExec_t exec = nullptr;
+};
+std::map<const void*, StepGraph> g_step;
+}  // namespace
+
+int dscale_verify_step_host_graph(void* ws, int n_bs, const int32_t* h_n_live, const float* h_scores,
+                                  const int32_t* h_draft_tokens, const int32_t* h_ctx_len,
+                                  const int32_t* h_block_table, int max_pages, int num_pages,
+                                  void* staging, const dscale_layer* layers, int n_layers,
+                                  int n_q_heads, int n_kv_heads, float sm_scale, const float* logits,
+                                  int64_t ld, int vocab, int32_t* h_accept_len, int32_t* h_next_anchor,
+                                  int32_t* h_out_tokens, int32_t* h_out_len, void* stream) {
+  auto plain = [&]() {
+    return dscale_verify_step_host(ws, n_bs, h_n_live, h_scores, h_draft_tokens, h_ctx_len, h_block_table,
+                                   max_pages, num_pages, staging, layers, n_layers, n_q_heads, n_kv_heads,
+                                   sm_scale, logits, ld, vocab, h_accept_len, h_next_anchor, h_out_tokens,
+                                   h_out_len, stream);
+  };
+  if (!ws || !layers || n_layers < 0) return DSCALE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) return DSCALE_ERR_CUDA;
+  if (cs != cudaStreamCaptureStatusNone) return plain();        // the caller is capturing: just record
+  if (st == nullptr || st == cudaStreamLegacy) return plain();  // the legacy default stream cannot capture
+
+  auto up = [](const void* p) { return reinterpret_cast<uintptr_t>(p); };
+  uint32_t scale_bits;
+  memcpy(&scale_bits, &sm_scale, 4);
+  std::vector<uintptr_t> key = {up(ws), (uintptr_t)n_bs, up(h_n_live), up(h_scores), up(h_draft_tokens),
+                                up(h_ctx_len), up(h_block_table), (uintptr_t)max_pages, (uintptr_t)num_pages,
+                                up(staging), (uintptr_t)n_layers, (uintptr_t)n_q_heads, (uintptr_t)n_kv_heads,
+                                (uintptr_t)scale_bits, up(logits), (uintptr_t)ld, (uintptr_t)vocab,
+                                up(h_accept_len), up(h_next_anchor), up(h_out_tokens), up(h_out_len)};
+  for (int l = 0; l < n_layers; ++l) {
+    key.push_back(up(layers[l].q)); key.push_back(up(layers[l].k_cache));
+    key.push_back(up(layers[l].v_cache)); key.push_back(up(layers[l].out));
+  }
+  std::lock_guard<std::mutex> lk(g_mu);
+  StepGraph& sg = g_step[ws];
+  if (!sg.exec || sg.key != key) {
+    if (sg.exec) { cudaGraphExecDestroy(sg.exec); sg.exec = nullptr; }
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return DSCALE_ERR_CUDA;
+    // plain() takes g_mu in its workspace lookups: release it around the capture body
+    g_mu.unlock();
+    const int rc = plain();
+    g_mu.lock();
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(st, &graph);
+    if (rc != DSCALE_OK || e != cudaSuccess || !graph) {
+      if (graph) cudaGraphDestroy(graph);
+      cudaGetLastError();
+      return rc != DSCALE_OK ? rc : DSCALE_ERR_CUDA;
+    }
+    const cudaError_t ei = cudaGraphInstantiate(&sg.exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ei != cudaSuccess) { sg.exec = nullptr; return DSCALE_ERR_CUDA; }
+    sg.key = key;
+  }
+  return cudaGraphLaunch(sg.exec, st) == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
 }
 
 int dscale_lm_head_accept(void* ws, int n_bs, const void* hidden, const void* weight, int hidden_dim,
