@@ -1,6 +1,7 @@
 // Acceptance-predictor front end: drafter logits and hidden states -> 1735
 // features -> 1735-64-15 perceptron -> predLogits ("Acceptance predictor"
-// paragraph, Eq. 4 and Eq. 5).  Four launches:
+// paragraph, Eq. 4 and Eq. 5).  Four launches (the hidden-state projection goes first and
+// overlaps with the logit stream):
 //
 //  pred_stream_kernel    the only pass over the drafter logits (15 N rows x V fp32,
 //                        292 MB at N = 32: an HBM stream).  A CTA of 16 warps owns
@@ -533,6 +534,7 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
 constexpr int kHidSlices = 4;                               // grid.y: 16 of the 64 outputs each
 
 __global__ void __launch_bounds__(kHidThreads) pred_hidden_kernel(FeatArgs a) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the logit stream may start now
   constexpr int kOut = kPredHid / kHidSlices;               // 16 outputs = 2 n-tiles
   __shared__ float red[kHidThreads / 32][16 * kOut];
   int n = *a.n_live;
@@ -723,16 +725,31 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   } else {
     tp = tz;                                            // never used: odd vocabularies stage the matrix by hand
   }
-  pred_stream_kernel<<<dim3(chunks, row_groups), kStreamThreads, kStreamSmem, stream>>>(sa, tz, tp);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
   FeatArgs fa{p.draft_logits, p.ld, p.vocab, p.n_live, p.n_bs,
               reinterpret_cast<const __nv_bfloat16*>(p.draft_hidden), p.hidden_dim,
               reinterpret_cast<const __nv_bfloat16*>(p.p_hidden), part, rowsum, chunks, feat};
-  pred_features_kernel<<<p.n_bs, kFeatThreads, 0, stream>>>(fa);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  // The hidden-state projection does not depend on the logit stream and is small: it goes
+  // first and lets its dependents start at once; the stream kernel is launched with
+  // programmatic stream serialisation and never waits for it, so the two overlap.  The
+  // feature merge and the perceptron are ordinary launches behind both.
   pred_hidden_kernel<<<dim3((kPredPos * p.n_bs + 15) / 16, kHidSlices), kHidThreads, 0, stream>>>(fa);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(chunks, row_groups);
+    cfg.blockDim = dim3(kStreamThreads);
+    cfg.dynamicSmemBytes = kStreamSmem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, pred_stream_kernel, sa, tz, tp);
+    if (e != cudaSuccess) return e;
+  }
+  pred_features_kernel<<<p.n_bs, kFeatThreads, 0, stream>>>(fa);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   MlpArgs ma{p.n_live, p.n_bs, feat, p.w1, p.b1, p.w2, p.b2, p.pred_logits, p.features_out};
