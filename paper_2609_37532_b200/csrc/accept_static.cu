@@ -91,7 +91,12 @@ __global__ void __launch_bounds__(kThreads) accept_static_kernel(Args a) {
   int* top1 = reinterpret_cast<int*>(a.scratch + kOffTop1);
   int N = *a.n_live;
   N = N < 1 ? 1 : (N > a.n_bs ? a.n_bs : N);
-  const int m_live = kHalfW * N;
+  // live packed rows = the end boundary of the last live request (Eq. 10): the
+  // lengths may come from an allocation under any budget, not only 8 N.  Clamped
+  // to the rows the launch and the scratch were sized for.
+  const int cap = kHalfW * a.n_bs;
+  int m_live = a.offset[N];
+  m_live = m_live < 1 ? 1 : (m_live > cap ? cap : m_live);
   const int s = blockIdx.y;
   if (s >= m_live) return;
   const int c = blockIdx.x, tid = threadIdx.x;
@@ -142,8 +147,10 @@ __global__ void __launch_bounds__(kThreads) accept_static_kernel(Args a) {
   if (tid < a.n_bs) {
     const int i = tid;
     int32_t* ot = a.out_tokens + i * kW;
-    if (i < N) {
-      const int ki = a.k[i], oi = a.offset[i];
+    // a request whose rows do not lie inside [0, m_live) (lengths and offsets are
+    // the caller's) gets the sentinel outputs instead of an out-of-range read
+    const int ki = i < N ? a.k[i] : 0, oi = i < N ? a.offset[i] : 0;
+    if (i < N && ki >= 1 && ki <= kW && oi >= 0 && oi + ki <= m_live) {
       int acc = 0;
       while (acc < ki - 1 && top1[oi + acc] == a.tokens[oi + acc + 1]) ++acc;
       const int nxt = top1[oi + acc];
