@@ -71,15 +71,43 @@ def oracle_attn(req, alloc, kc, vc, qp, dtype=np.float32):
                           req["n_live"], cfg.n_q_heads, cfg.n_kv_heads, SCALE, dtype=dtype)
 
 
+ROW_REL_L2 = 8e-3      # per (row, head) output vector: ||gpu - ref||_2 <= ROW_REL_L2 ||ref||_2 + ROW_ABS_L2
+ROW_ABS_L2 = 2e-4
+
+
+def attn_stats(got: np.ndarray, ref: np.ndarray) -> dict:
+    """Error figures of an attention output against the oracle: max abs, max rel over
+    |ref| > 1e-2, ||d||_2 / ||ref||_2 over everything, and the worst per-(row, head) vector."""
+    err = np.abs(got - ref)
+    big = np.abs(ref) > 1e-2
+    num = np.sqrt((err.astype(np.float64) ** 2).sum(axis=-1))
+    den = np.sqrt((ref.astype(np.float64) ** 2).sum(axis=-1))
+    row_excess = num - (ROW_REL_L2 * den + ROW_ABS_L2)
+    return dict(max_abs=float(err.max()),
+                max_rel=float((err[big] / np.abs(ref[big])).max()) if big.any() else 0.0,
+                rel_l2=float(np.sqrt((num ** 2).sum() / max((den ** 2).sum(), 1e-300))),
+                worst_row_rel_l2=float((num / np.maximum(den, 1e-30))[den > 1e-3].max()) if (den > 1e-3).any() else 0.0,
+                row_excess=row_excess)
+
+
 def attn_close(got_bf16: torch.Tensor, ref: np.ndarray, atol=1e-2, rtol=1e-2):
-    """Pass iff |gpu - ref| <= atol + rtol |ref| for every element; returns
-    (ok, max_abs, worst_index) so a failure can say where."""
+    """The parity bar for bf16 attention outputs.  Per element: |gpu - ref| <= max(atol, rtol |ref|)
+    (1e-2 absolute or 1e-2 relative, whichever is larger: tighter than the sum of the two).
+    Per (row, head) output vector: ||gpu - ref||_2 <= 8e-3 ||ref||_2 + 2e-4.  The vector bound is the
+    sharp one: with N(0,1) inputs and thousands of keys an output element is a few 1e-2, bf16
+    rounding of the probabilities and of the result costs about 2e-3 of the vector's norm, while a
+    dropped 16-key page shifts a vector by several per cent of its norm.
+    Returns (ok, max_abs, worst_index) so a failure can say where."""
     got = got_bf16.float().cpu().numpy()
     if not np.isfinite(got).all():
         bad = np.argwhere(~np.isfinite(got))[0]
         return False, float("nan"), tuple(bad)
     err = np.abs(got - ref)
-    lim = atol + rtol * np.abs(ref)
+    lim = np.maximum(atol, rtol * np.abs(ref))
+    st = attn_stats(got, ref)
+    if (st["row_excess"] > 0).any():
+        worst = np.unravel_index(np.argmax(st["row_excess"]), st["row_excess"].shape)
+        return False, float(err.max()), tuple(int(x) for x in worst) + (-1,)
     worst = np.unravel_index(np.argmax(err - lim), err.shape)
     return bool((err <= lim).all()), float(err.max()), tuple(int(x) for x in worst)
 
