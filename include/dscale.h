@@ -13,7 +13,12 @@
  * General rules
  * -------------
  *  - Unless a parameter is marked HOST, every pointer is a DEVICE pointer that
- *    the caller owns; the library never allocates, frees or synchronises.
+ *    the caller owns.  No call allocates or frees DEVICE memory, and none
+ *    synchronises.  Host-side state the library does keep: one registry entry
+ *    per initialised workspace, tensor-map descriptors keyed on the q / K / V
+ *    addresses it has seen (a few hundred bytes each), and, for
+ *    dscale_verify_step_host_graph only, one instantiated CUDA graph per
+ *    workspace (driver memory).  dscale_workspace_destroy drops all of it.
  *  - Every call only enqueues kernels on `stream` (a cudaStream_t passed as
  *    void*).  All shapes are fixed by the arguments, every data-dependent
  *    quantity (N, lengths, offsets, context lengths) is read on the device,
@@ -104,6 +109,16 @@ size_t dscale_workspace_bytes(int n_bs, int n_q_heads, int n_kv_heads, int head_
  */
 int dscale_workspace_init(void* ws, size_t bytes, int n_bs, int n_q_heads, int n_kv_heads,
                           int head_dim, int num_sms, void* stream);
+
+/*
+ * Forget a workspace: removes its registry entry, destroys the step graph that
+ * dscale_verify_step_host_graph cached for it, and drops the cached tensor-map
+ * descriptors (they are keyed on buffer addresses that the caller is about to
+ * free or reuse).  HOST call; call it before freeing the workspace memory, with
+ * no work on the workspace in flight.  The device memory itself stays the
+ * caller's.  Returns DSCALE_ERR_WORKSPACE for a pointer that is not registered.
+ */
+int dscale_workspace_destroy(void* ws);
 
 /*
  * DVL allocation and flat-pack (Algorithm 1 from its second line; Eq. 6, 7, 9, 10, 11).
@@ -347,8 +362,11 @@ int dscale_predict_scores(void* ws, int n_bs, const int32_t* n_live, const float
  *   outputs   as in dscale_accept
  * Logits must be finite.  Probabilities are evaluated in fp32; a draw whose
  * target falls within rounding of a boundary of the cumulative sum may return
- * the neighbouring token.
+ * the neighbouring token.  vocab <= DSCALE_SAMPLING_MAX_VOCAB (the draw kernel
+ * keeps one partial sum per 1024 tokens in a fixed table), otherwise
+ * DSCALE_ERR_TOO_LARGE and nothing is enqueued.
  */
+#define DSCALE_SAMPLING_MAX_VOCAB (1 << 20)
 int dscale_accept_sampling(void* ws, int n_bs, const float* logits, int64_t ld, int vocab,
                            float temperature, const float* u_accept, const float* u_draw,
                            int32_t* accept_len, int32_t* next_anchor, int32_t* out_tokens,
@@ -367,8 +385,13 @@ int dscale_accept_sampling(void* ws, int n_bs, const float* logits, int64_t ld, 
  *
  *   n_live [1], k [n_bs], offset [n_bs + 1], tokens [8 n_bs]   int32, device:
  *         as produced by dscale_alloc_verify (workspace fields N_LIVE, K,
- *         OFFSET, TOKENS) or by the caller
+ *         OFFSET, TOKENS) or by the caller, under any budget and block width
+ *         that dscale_alloc_verify_ex serves: the number of live packed rows is
+ *         read on the device as offset[N] (clamped to 8 n_bs)
  *   logits, ld, vocab and the four outputs: as in dscale_accept
+ * A live request whose rows do not lie inside the live packed rows (k outside
+ * 1..16, a negative offset, offset + k beyond offset[N]) gets the outputs of a
+ * sentinel (length 0, next anchor -1); there is no status word in this call.
  *
  * Limits and rules: n_bs <= DSCALE_ACCEPT_STATIC_MAX_NBS, otherwise
  * DSCALE_ERR_TOO_LARGE is returned and nothing is enqueued.  All calls on a GPU

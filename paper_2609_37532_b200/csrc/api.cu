@@ -15,6 +15,7 @@ cudaError_t attn_simt_prepare();
 cudaError_t attn_tc_prepare();
 cudaError_t attn_padded_prepare();
 cudaError_t lm_head_prepare();
+void attn_tc_forget_maps();
 }
 
 namespace {
@@ -73,6 +74,33 @@ int dscale_workspace_init(void* ws, size_t bytes, int n_bs, int n_q_heads, int n
   if (predictor_prepare() != cudaSuccess) return DSCALE_ERR_CUDA;
   std::lock_guard<std::mutex> lk(g_mu);
   g_ws[ws] = WsInfo{bytes, n_bs, n_q_heads, n_kv_heads, num_sms};
+  return DSCALE_OK;
+}
+
+namespace {
+struct StepGraph {   // one instantiated graph of the host-driven step per workspace, keyed by every argument
+  std::vector<uintptr_t> key;
+  cudaGraphExec_t exec = nullptr;
+};
+std::map<const void*, StepGraph> g_step;
+}  // namespace
+
+int dscale_workspace_destroy(void* ws) {
+  if (!ws) return DSCALE_ERR_INVALID_ARG;
+  cudaGraphExec_t exec = nullptr;
+  {
+    std::lock_guard<std::mutex> lk(g_mu);
+    auto it = g_ws.find(ws);
+    if (it == g_ws.end()) return DSCALE_ERR_WORKSPACE;
+    g_ws.erase(it);
+    auto sg = g_step.find(ws);
+    if (sg != g_step.end()) { exec = sg->second.exec; g_step.erase(sg); }
+  }
+  if (exec) cudaGraphExecDestroy(exec);
+  // tensor-map descriptors are keyed on the q / K / V addresses, which the caller
+  // is about to free or reuse along with the workspace: drop them all (they are
+  // re-encoded on the next call that needs one)
+  attn_tc_forget_maps();
   return DSCALE_OK;
 }
 
@@ -261,15 +289,6 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
   return DSCALE_OK;
 }
 
-namespace {
-// one instantiated graph of the host-driven step per workspace, keyed by every argument
-struct StepGraph {
-  std::vector<uintptr_t> key;
-  cudaGraphExec_t exec = nullptr;
-};
-std::map<const void*, StepGraph> g_step;
-}  // namespace
-
 int dscale_verify_step_host_graph(void* ws, int n_bs, const int32_t* h_n_live, const float* h_scores,
                                   const int32_t* h_draft_tokens, const int32_t* h_ctx_len,
                                   const int32_t* h_block_table, int max_pages, int num_pages,
@@ -302,15 +321,17 @@ int dscale_verify_step_host_graph(void* ws, int n_bs, const int32_t* h_n_live, c
     key.push_back(up(layers[l].q)); key.push_back(up(layers[l].k_cache));
     key.push_back(up(layers[l].v_cache)); key.push_back(up(layers[l].out));
   }
-  std::lock_guard<std::mutex> lk(g_mu);
-  StepGraph& sg = g_step[ws];
-  if (!sg.exec || sg.key != key) {
-    if (sg.exec) { cudaGraphExecDestroy(sg.exec); sg.exec = nullptr; }
+  cudaGraphExec_t exec = nullptr;
+  {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (g_ws.find(ws) == g_ws.end()) return DSCALE_ERR_WORKSPACE;
+    auto it = g_step.find(ws);
+    if (it != g_step.end() && it->second.exec && it->second.key == key) exec = it->second.exec;
+  }
+  if (!exec) {
+    // capture outside the registry lock: the stage calls inside plain() take it themselves
     if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return DSCALE_ERR_CUDA;
-    // plain() takes g_mu in its workspace lookups: release it around the capture body
-    g_mu.unlock();
     const int rc = plain();
-    g_mu.lock();
     cudaGraph_t graph = nullptr;
     const cudaError_t e = cudaStreamEndCapture(st, &graph);
     if (rc != DSCALE_OK || e != cudaSuccess || !graph) {
@@ -318,12 +339,20 @@ int dscale_verify_step_host_graph(void* ws, int n_bs, const int32_t* h_n_live, c
       cudaGetLastError();
       return rc != DSCALE_OK ? rc : DSCALE_ERR_CUDA;
     }
-    const cudaError_t ei = cudaGraphInstantiate(&sg.exec, graph, 0);
+    const cudaError_t ei = cudaGraphInstantiate(&exec, graph, 0);
     cudaGraphDestroy(graph);
-    if (ei != cudaSuccess) { sg.exec = nullptr; return DSCALE_ERR_CUDA; }
-    sg.key = key;
+    if (ei != cudaSuccess || !exec) return DSCALE_ERR_CUDA;
+    cudaGraphExec_t old = nullptr;
+    {
+      std::lock_guard<std::mutex> lk(g_mu);
+      StepGraph& sg = g_step[ws];
+      old = sg.exec;
+      sg.exec = exec;
+      sg.key = key;
+    }
+    if (old) cudaGraphExecDestroy(old);
   }
-  return cudaGraphLaunch(sg.exec, st) == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
+  return cudaGraphLaunch(exec, st) == cudaSuccess ? DSCALE_OK : DSCALE_ERR_CUDA;
 }
 
 int dscale_lm_head_accept(void* ws, int n_bs, const void* hidden, const void* weight, int hidden_dim,
@@ -368,6 +397,7 @@ int dscale_accept_sampling(void* ws, int n_bs, const float* logits, int64_t ld, 
     return DSCALE_ERR_INVALID_ARG;
   if (vocab < 1 || ld < vocab || (ld % 4) != 0 || !aligned(logits, 16) || !(temperature > 0.0f))
     return DSCALE_ERR_INVALID_ARG;
+  if (vocab > DSCALE_SAMPLING_MAX_VOCAB) return DSCALE_ERR_TOO_LARGE;   // the draw kernel's group table
   WsInfo info;
   if (!lookup(ws, n_bs, &info)) return DSCALE_ERR_WORKSPACE;
   SampleArgs a{ws, n_bs, logits, ld, vocab, temperature, u_accept, u_draw, accept_len, next_anchor,

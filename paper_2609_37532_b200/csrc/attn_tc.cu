@@ -909,6 +909,12 @@ bool q_map(const void* ptr, int n_q, int rows, CUtensorMap* out) {
 
 }  // namespace
 
+void attn_tc_forget_maps() {
+  std::lock_guard<std::mutex> lk(g_map_mu);
+  g_kv_maps.clear();
+  g_q_maps.clear();
+}
+
 cudaError_t attn_tc_prepare() {
   return cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               kSmemBytes);

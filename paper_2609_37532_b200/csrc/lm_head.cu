@@ -24,6 +24,7 @@
 // order -- so equal maxima resolve to the lowest index -- and runs the acceptance
 // loop of the "Prefix verifier" paragraph.
 #include <climits>
+#include <mutex>
 
 #include "kernels.cuh"
 #include "tc_ptx.cuh"
@@ -644,10 +645,17 @@ PairShape plan_pair(int n_bs, int vocab, int pairs) {
 // CTA pairs that can be resident at once with the ring at its largest (one CTA
 // per SM either way); a grid beyond it would run a second, nearly empty wave.
 int resident_pairs(int num_ctas) {
-  static int cached = -1;
-  if (cached < 0) {
+  // The answer depends on the device (SM count, shared memory), not on the grid asked
+  // about, so it is kept per device; a failed query is not kept.
+  static std::mutex mu;
+  static int cached[64];
+  static bool have[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  std::lock_guard<std::mutex> lk(mu);
+  if (!have[dev]) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((num_ctas / 2) * 2);
+    cfg.gridDim = dim3(2);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = 224 * 1024;
     cudaLaunchAttribute at[1];
@@ -655,11 +663,12 @@ int resident_pairs(int num_ctas) {
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, lm_head_pair_kernel<1>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-    cached = n;
+    if (cudaOccupancyMaxActiveClusters(&n, lm_head_pair_kernel<1>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    cached[dev] = n;
+    have[dev] = true;
   }
   const int want = num_ctas / 2;
-  return cached < want ? cached : want;
+  return cached[dev] < want ? cached[dev] : want;
 }
 
 }  // namespace

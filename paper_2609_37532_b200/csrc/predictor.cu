@@ -211,6 +211,8 @@ __device__ __forceinline__ void row_update2(RowStat& a, RowStat& b, float4 za, f
   }
 }
 
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __global__ void __launch_bounds__(kStreamThreads, 1)
 pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const __grid_constant__ CUtensorMap tm_p) {
   extern __shared__ unsigned char smem_raw[];
@@ -230,11 +232,11 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
   n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
   const int live_rows = kPredPos * n;
   const int row0 = blockIdx.y * kRowsPerCta;
-  if (row0 >= live_rows) return;
+  if (row0 >= live_rows) { pdl_wait(); return; }
   const int chunk = blockIdx.x;
   const int col_lo = chunk * a.chunk_len;
   const int col_hi = min(a.vocab, col_lo + a.chunk_len);
-  if (col_lo >= col_hi) return;
+  if (col_lo >= col_hi) { pdl_wait(); return; }
   const int n_sub = (col_hi - col_lo + kSub - 1) / kSub;
 
   // warp w owns rows w and w + 16 of the CTA's 32 (one in each 16-row MMA tile)
@@ -376,6 +378,7 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
     // status word and leave.
     if (tid == 0) atomicOr(a.status, 8 /*TIMEOUT*/);
     __syncthreads();
+    pdl_wait();
     return;
   }
 
@@ -430,6 +433,12 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
     for (int o = 8; o > 0; o >>= 1) p_rowsum += __shfl_xor_sync(0xffffffffu, p_rowsum, o);
     if (pq == 0) a.rowsum[chunk * kPredLog + pj] = p_rowsum;
   }
+  // This grid was allowed to start before the hidden-projection kernel ahead of it in
+  // the stream had finished (it reads nothing that kernel writes).  The kernels behind
+  // this one do read it, and they are ordered only behind this grid: waiting here, as
+  // the last thing every CTA does, makes this grid's completion imply the completion
+  // and memory flush of that kernel.
+  pdl_wait();
 }
 
 // ---------------------------------------------------------------------------
@@ -730,8 +739,9 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
               reinterpret_cast<const __nv_bfloat16*>(p.p_hidden), part, rowsum, chunks, feat};
   // The hidden-state projection does not depend on the logit stream and is small: it goes
   // first and lets its dependents start at once; the stream kernel is launched with
-  // programmatic stream serialisation and never waits for it, so the two overlap.  The
-  // feature merge and the perceptron are ordinary launches behind both.
+  // programmatic stream serialisation and waits for it only as its last action, so the two
+  // overlap.  The feature merge and the perceptron are ordinary launches behind the
+  // stream kernel, whose completion then implies the hidden projection's.
   pred_hidden_kernel<<<dim3((kPredPos * p.n_bs + 15) / 16, kHidSlices), kHidThreads, 0, stream>>>(fa);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
