@@ -7,9 +7,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# DSCALE_LIB points the binding at another build of the same library (for
-# example one compiled with -DDSCALE_TRACE); the default is the in-tree build.
-_LIB_PATH = os.environ.get("DSCALE_LIB") or os.path.join(_HERE, "libdscale.so")
+_LIB_PATH = os.path.join(_HERE, "libdscale.so")
 
 if not os.path.exists(_LIB_PATH):
     raise ImportError(
@@ -23,6 +21,8 @@ lib.dscale_workspace_bytes.restype = _sz
 lib.dscale_workspace_bytes.argtypes = [_i, _i, _i, _i, _i]
 lib.dscale_workspace_init.restype = _i
 lib.dscale_workspace_init.argtypes = [_vp, _sz, _i, _i, _i, _i, _i, _vp]
+lib.dscale_workspace_destroy.restype = _i
+lib.dscale_workspace_destroy.argtypes = [_vp]
 lib.dscale_alloc_verify.restype = _i
 lib.dscale_alloc_verify.argtypes = [_vp, _i, _vp, _vp, _i, _vp, _vp, _vp, _i, _i, _vp]
 lib.dscale_alloc_verify_ex.restype = _i
@@ -112,6 +112,19 @@ class VerifyWorkspace:
             _check(lib.dscale_workspace_init(C.c_void_p(self.ptr), nbytes, n_bs, n_q_heads,
                                              n_kv_heads, head_dim, self.num_sms, _stream()),
                    "dscale_workspace_init")
+
+    def close(self):
+        """Forget the workspace in the library (registry entry, cached step graph, tensor
+        maps) and release its memory.  No work on it may be in flight."""
+        if self.ptr:
+            lib.dscale_workspace_destroy(C.c_void_p(self.ptr))
+            self.ptr, self.buf = 0, None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
     def field(self, name: str) -> torch.Tensor:
         """int32 view of a workspace section (shares memory with the workspace)."""

@@ -201,6 +201,38 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
     wref[t] = page * kPage + pos % kPage;
     wreq[t] = -1;
   }
+  // ---- attention schedule: slice c of the persistent grid starts at linear key tile
+  // slice_tab[c] (request-major, then kv-head, then tile).  Slices have equal cost; the
+  // last two CTAs of a launch, which start last, get three tiles and one tile less.
+  // Small tile counts (under 8 per CTA) are cut by count, and with fewer tiles than CTAs
+  // the first T CTAs get one tile each.
+  for (int cta = t; cta <= a.num_ctas; cta += blockDim.x) {
+    const int n_kv = a.n_kv_heads;
+    const long long T = (long long)sTilePre[kMaxNbs] * n_kv;
+    const long long C = T < a.num_ctas ? T : a.num_ctas;
+    long long tile = T;
+    if (cta < C) {
+      const bool by_count = T < 8 * C;
+      const bool skew = C >= 8 && T / C >= 24;
+      const int unit = by_count ? 1 : kTileCostSmall;
+      long long W = 0;
+      for (int r = 0; r < N; ++r) {
+        const int w = by_count ? 1 : (sK[r] > 8 ? kTileCostBig : kTileCostSmall);
+        W += (long long)(sTilePre[r + 1] - sTilePre[r]) * w * n_kv;
+      }
+      const long long d1 = skew ? 3 * unit : 0, d2 = skew ? unit : 0;
+      const long long Wv = W + d1 + d2;                      // equal shares of a slightly longer list ...
+      const long long x = (cta == C - 1) ? (C - 1) * Wv / C - d2 : (long long)cta * Wv / C;   // ... the last two give some back
+      long long acc = 0;
+      for (int r = 0; r < N; ++r) {
+        const int w = by_count ? 1 : (sK[r] > 8 ? kTileCostBig : kTileCostSmall);
+        const long long rc = (long long)(sTilePre[r + 1] - sTilePre[r]) * w * n_kv;
+        if (x < acc + rc) { tile = (long long)sTilePre[r] * n_kv + (x - acc) / w; break; }
+        acc += rc;
+      }
+    }
+    ws_ptr<int>(a.ws, L.slice_tab)[cta] = (int)tile;
+  }
   __syncthreads();
   if (t == 0) {
     hdr[H_N_LIVE] = N;

@@ -2,7 +2,7 @@
 //
 // Shape of the work.  Per live request i and kv-head g the query tile is the
 // GQA group's 4 q-heads x the k_i <= 16 live window rows = at most 64 rows:
-// exactly one M = 64 tcgen05 tile (row m = 4 j + h_local), instead of the
+// exactly one M = 64 tcgen05 tile (row m = 16 h_local + j), instead of the
 // 128-row prefill tile that would leave 112 masked rows per request and head
 // (Eq. 2).  Keys and values are streamed once per kv-head in tiles of 128
 // tokens (8 pages).  The kernel is HBM-bound; the tensor cores only have to
@@ -23,21 +23,30 @@
 // The grid and every address are independent of the lengths, so a captured
 // launch replays at any mix of lengths.
 //
-// Pipeline inside a CTA (224 threads):
-//   warp 4     producer: per tile, 16 + 16 TMA box copies (one 16-token page
-//              x 64 columns each, 128-byte swizzle) of K then V into a 5-deep
-//              ring of 32 KB slots; page ids are fetched one tile ahead.
-//   warp 5     one thread issues tcgen05.mma: S = Q K^T (M64 N128 K128, bf16 in,
+// Pipeline inside a CTA (352 threads):
+//   warp 8     producer: per tile, 16 TMA box copies of K (a 64-column half of one
+//              16-token page each, 2 KB) and 8 of V (a whole page-head, 4 KB), 128-byte
+//              swizzle, into a 5-deep ring of 32 KB slots; page ids are fetched one
+//              tile ahead.  Both the copy engine and the single MMA-issuing thread pay
+//              about 100 SM cycles per instruction whatever its size, and once the SM
+//              clock drops under the power cap either count can bound the stream:
+//              24 copies and 16 products per tile keep both below the memory time
+//              (32 + 16 made the copies the bound, 16 + 24 the products).
+//   warp 9     one thread issues tcgen05.mma: S = Q K^T (M64 N128 K128, bf16 in,
 //              fp32 in TMEM) for tile t, then O_t = P_{t-1} V_{t-1}; completion
 //              is signalled with tcgen05.commit on mbarriers.
-//   warps 0-3  softmax: warp w owns tile rows 16 w .. 16 w + 15 (TMEM lanes 32 w ..
-//              32 w + 15); tcgen05.ld.16x256b spreads them over all 32 lanes (a
-//              quad of threads per row).  They keep the running max / sum and
+//   warps 0-7  softmax.  Tile rows are head-major (m = 16 h_local + j), so q-head
+//              h_local sits in TMEM lanes 32 h_local .. 32 h_local + 15, which
+//              warps h_local and h_local + 4 may read.  Warp h_local takes window
+//              rows j = 0..7, warp h_local + 4 rows j = 8..15: a thread owns one
+//              row together with the three other threads of its quad
+//              (tcgen05.ld.16x256b), and a request with k_i <= 8 leaves the
+//              second group of warps idle.  They keep the running max / sum and
 //              write P as bf16 into swizzled shared memory for the second MMA.  O stays in
 //              TMEM for a whole run of tiles (the second MMA accumulates onto
 //              it); it is only rescaled in place when a row maximum outgrows its
 //              reference by 2^8, and read back once per run for the epilogue.
-//   warp 6     publisher: fence + ticket for the first run's partial.
+//   warp 10    publisher: fence + ticket for the first run's partial.
 // S is triple-buffered in TMEM (3 x 128 columns) next to O (128 columns), P and
 // Q are double-buffered in shared memory; the MMA thread issues whichever of the
 // two products is ready, scores up to two tiles ahead of the softmax.
@@ -58,17 +67,19 @@ namespace dscale {
 
 namespace {
 
-constexpr int kThreads = 224;
-constexpr int kSoftmaxThreads = 128;
+constexpr int kThreads = 352;
+constexpr int kSoftmaxThreads = 256;
+constexpr int kWarpProducer = 8, kWarpMma = 9, kWarpPublisher = 10;
 #ifndef DSCALE_STAGES
 #define DSCALE_STAGES 5
 #endif
 constexpr int kStages = DSCALE_STAGES;
 constexpr int kSlotBytes = kTileTok * kD * 2;           // 32 KB: one K or V tile
-constexpr int kHalfSlot = kSlotBytes / 2;               // one 64-column half [128 tok][128 B]
+constexpr int kHalfSlot = kSlotBytes / 2;               // K tile: one 64-column half [128 tok][128 B]
+constexpr int kPageBytes = kPage * kD * 2;              // V tile: 4 KB per page-head = one TMA box
+constexpr int kPageHalf = kPageBytes / 2;               // a page's 64-column half [16 tok][128 B]
 constexpr int kQBytes = kTcRows * kD * 2;               // 16 KB
 constexpr int kPBytes = kTcRows * kTileTok * 2;         // 16 KB
-constexpr int kPageBoxBytes = kPage * 64 * 2;           // 2 KB per TMA box
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;                                 // 2 x 16 KB
@@ -77,8 +88,10 @@ constexpr int kOffKV = kOffP + 2 * kPBytes;              // 5 x 32 KB
 constexpr int kOffBar = kOffKV + kStages * kSlotBytes;   // mbarriers
 constexpr int kNumBars = 2 * kStages + 2 + 2 + 3 + 2 + 2 + 5;
 constexpr int kOffMisc = kOffBar + 8 * 32;               // tmem base, abort flag, tickets
-constexpr int kOffTile = kOffMisc + 48;                  // tile prefix, kMaxNbs + 1 ints
-constexpr int kSmemUse = kOffTile + (kMaxNbs + 1) * 4 + 12;
+constexpr int kOffTile = kOffMisc + 64;                  // tile prefix, kMaxNbs + 1 ints
+constexpr int kOffSlice = kOffTile + (kMaxNbs + 1) * 4 + 12;   // slice starts, up to kMaxCtas + 1 ints
+constexpr int kMaxCtas = 255;
+constexpr int kSmemUse = kOffSlice + (kMaxCtas + 1) * 4;
 constexpr int kSmemBytes = kSmemUse + 1024;              // slack for base alignment
 static_assert(kNumBars <= 32, "barrier area");
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
@@ -93,10 +106,11 @@ enum Bar { B_KV_FULL = 0, B_KV_EMPTY = kStages, B_Q_FULL = 2 * kStages, B_Q_EMPT
 
 // instruction descriptor: bf16 x bf16 -> fp32, M = 64, N = 128; B is K-major
 // for S = Q K^T and MN-major (tokens are the K dimension) for O = P V
-constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) |
-                                ((64u >> 4) << 24);
-constexpr uint32_t kIdescS = kIdescBase;
-constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);
+constexpr uint32_t idesc(uint32_t n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((64u >> 4) << 24);
+}
+constexpr uint32_t kIdescS = idesc(128);
+constexpr uint32_t kIdescPV = idesc(128) | (1u << 16);
 
 #ifdef DSCALE_TRACE
 __device__ __forceinline__ unsigned long long gtime() {
@@ -137,7 +151,9 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   volatile int* s_fast = reinterpret_cast<volatile int*>(sm + kOffMisc + 20);      // partner partials in smem
   volatile int* s_head_last = reinterpret_cast<volatile int*>(sm + kOffMisc + 24); // publisher took the last ticket
   volatile int* s_dummy = reinterpret_cast<volatile int*>(sm + kOffMisc + 16);
+  volatile int* s_lock = reinterpret_cast<volatile int*>(sm + kOffMisc + 32);     // one per q-head: O rescale turn
   int* s_tile = reinterpret_cast<int*>(sm + kOffTile);
+  int* s_slice = reinterpret_cast<int*>(sm + kOffSlice);
   auto bar = [&](int b) { return base + kOffBar + 8u * b; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -163,14 +179,15 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     mbar_init(bar(B_MERGE), 1);
     *s_abort = 0;
     *s_dummy = 0;
+    for (int x = 0; x < 4; ++x) s_lock[x] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 5) {
+  if (warp == kWarpMma) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
                  ::"r"(smem_u32(s_tmem)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (warp == 4 && lane == 0) {
+  if (warp == kWarpProducer && lane == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
@@ -186,21 +203,23 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   // as soon as SMs free up.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   for (int x = tid; x <= n_bs; x += kThreads) s_tile[x] = ws_ptr<int>(a.ws, L.tile_prefix)[x];
+  for (int x = tid; x <= (int)gridDim.x; x += kThreads) s_slice[x] = ws_ptr<int>(a.ws, L.slice_tab)[x];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
-  if (warp != 4) asm volatile("griddepcontrol.wait;" ::: "memory");   // the producer waits later
+  if (warp != kWarpProducer) asm volatile("griddepcontrol.wait;" ::: "memory");   // the producer waits later
 
   const long long T = (long long)s_tile[n_bs] * n_kv;
   // with fewer tiles than CTAs only the first T CTAs get a (one-tile) slice, so
   // that every CTA in [0, C) has work and the per-pair contributor count is exact
   const int C = (int)min((long long)gridDim.x, T);
-  const long long sl_begin = c < C ? slice_begin(c, T, C) : 0;
-  const long long sl_end = c < C ? slice_begin(c + 1, T, C) : 0;
+  const long long sl_begin = c < C ? s_slice[c] : 0;
+  const long long sl_end = c < C ? s_slice[c + 1] : 0;
+  auto cta_of = [&](long long Lt) { return cta_of_tab(s_slice, C, Lt); };
   const int* kv_len = ws_ptr<int>(a.ws, L.kv_len);
 
-  if (warp == 4) {
+  if (warp == kWarpProducer) {
     // ===================================================== TMA producer warp
     Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
     Segment sg;
@@ -208,10 +227,15 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     int seg = 0;
     bool ok = true;
     bool waited = false;       // griddepcontrol.wait done
-    // lane l copies page l / 2, column half l % 2 (lanes 0..15)
-    const int pg_l = lane >> 1, half = lane & 1;
+    // V: lane l < 8 copies page l of the tile as one 4 KB box.  K: lanes l and l + 8 copy
+    // the two 64-column halves of page l as 2 KB boxes (see the shared-memory layouts below).
+    const int pg_l = lane & 7, k_half = lane >> 3;
     // K/V are read exactly once per launch: mark them evict-first in L2
     const uint64_t kv_policy = make_policy_evict_first();
+#ifdef DSCALE_TRACE
+    long long prod_wait = 0, prod_fetch = 0;
+    const long long prod_t0 = clock64();
+#endif
     while (ok && sch.next(sg)) {
       const int qb = seg & 1;
       const int len = kv_len[sg.i];
@@ -231,13 +255,22 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
         for (int which = 0; which < 2; ++which, ++u) {
           const int slot = u % kStages;
+#ifdef DSCALE_TRACE
+          const long long pw0 = clock64();
+#endif
           if (!mbar_wait(bar(B_KV_EMPTY + slot), ((u / kStages) & 1) ^ 1, s_abort)) return false;
-          if (lane == 0) mbar_expect_tx(bar(B_KV_FULL + slot), n_pages * 2 * kPageBoxBytes);
+#ifdef DSCALE_TRACE
+          prod_wait += clock64() - pw0;
+#endif
+          if (lane == 0) mbar_expect_tx(bar(B_KV_FULL + slot), n_pages * kPageBytes);
           __syncwarp();
-          if (lane < 16 && pg_l < n_pages) {
-            tma_load_5d_hint(base + kOffKV + slot * kSlotBytes + half * kHalfSlot + pg_l * kPageBoxBytes,
-                             which == 0 ? &tm_k : &tm_v, bar(B_KV_FULL + slot), 0, half, 0, sg.g, page,
-                             kv_policy);
+          if (which == 0) {
+            if (lane < 16 && pg_l < n_pages)
+              tma_load_5d_hint(base + kOffKV + slot * kSlotBytes + k_half * kHalfSlot + pg_l * kPageHalf,
+                               &tm_k, bar(B_KV_FULL + slot), 0, k_half, 0, sg.g, page, kv_policy);
+          } else if (lane < 8 && pg_l < n_pages) {
+            tma_load_5d_hint(base + kOffKV + slot * kSlotBytes + pg_l * kPageBytes,
+                             &tm_v, bar(B_KV_FULL + slot), 0, 0, 0, sg.g, page, kv_policy);
           }
         }
         return true;
@@ -263,14 +296,20 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       if (!ok) break;
       if (lane == 0) {
         mbar_expect_tx(bar(B_Q_FULL + qb), kQBytes);
-        tma_load_4d(base + kOffQ + qb * kQBytes, &tm_q, bar(B_Q_FULL + qb), 0, 0, sg.g * 4, row0);
+        tma_load_4d(base + kOffQ + qb * kQBytes, &tm_q, bar(B_Q_FULL + qb), 0, 0, row0, sg.g * 4);
         tma_load_4d(base + kOffQ + qb * kQBytes + kQBytes / 2, &tm_q, bar(B_Q_FULL + qb), 0, 1,
-                    sg.g * 4, row0);
+                    row0, sg.g * 4);
       }
       int page_next = t_first < sg.t1 ? fetch_page(t_first) : 0;
       for (int t = t_first; t < sg.t1 && ok; ++t) {
         const int page = page_next;
+#ifdef DSCALE_TRACE
+        const long long pf0 = clock64();
+#endif
         if (t + 1 < sg.t1) page_next = fetch_page(t + 1);
+#ifdef DSCALE_TRACE
+        prod_fetch += clock64() - pf0;
+#endif
         ok = issue_tile(t, page);
       }
       if (ok && run_kind(sg, sch.more()) == RUN_TAIL) {
@@ -280,7 +319,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         // tiles, so that the softmax warps can finish the pair without a single
         // global round trip.
         const long long p0 = ((long long)s_tile[sg.i] * n_kv) + (long long)sg.g * sg.n_tiles;
-        const int c_hi = cta_of(p0 + sg.n_tiles - 1, T, C);
+        const int c_hi = cta_of(p0 + sg.n_tiles - 1);
         const int others = c_hi - c;                       // this CTA holds the pair's first tiles
         int fast = 0;
         if (others <= kMaxFastPartners) {
@@ -312,13 +351,17 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       ++seg;
     }
     if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef DSCALE_TRACE
+    if (lane == 0) { unsigned long long* trp = ws_ptr<unsigned long long>(a.ws, L.trace) + (size_t)c * 64;
+                     trp[40] = prod_wait; trp[41] = clock64() - prod_t0; trp[45] = prod_fetch; }
+#endif
     // on an aborted run, let the copies already issued land before the CTA's
     // shared memory is released (bounded, like every other wait)
     if (!ok) {
       for (unsigned v = (u > kStages ? u - kStages : 0); v < u; ++v)
         mbar_wait(bar(B_KV_FULL + v % kStages), (v / kStages) & 1, s_dummy);
     }
-  } else if (warp == 5) {
+  } else if (warp == kWarpMma) {
     // ============================================================ MMA issuer
     if (lane == 0) {
       // Event-driven issue.  S = Q K^T of tile x goes into TMEM buffer x % 3 as soon
@@ -335,6 +378,10 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       unsigned run_start_mask = 0;               // bit (x % 4): tile x starts a run
       bool ok = true;
       long long t_idle = clock64();
+#ifdef DSCALE_TRACE
+      long long mma_loops = 0, mma_idle = 0;
+      const long long mma_t0 = clock64();
+#endif
       while (ok && next_pv < total) {
         bool progressed = false;
         // ---- O += P V for the oldest tile whose P is ready
@@ -352,8 +399,9 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
             for (int kk = 0; kk < kTileTok / 16; ++kk) {
               // A = P [64 rows][128 tok] K-major: 64-token blocks of 8 KB, 32 B per 16 tokens
               const uint64_t ad = smem_desc(p_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
-              // B = V [128 tok][128 d] with d contiguous: MN-major, 16 tokens = 2 KB
-              const uint64_t bd = smem_desc(v_base + kk * (16 * 128), kHalfSlot, 1024);
+              // B = V, MN-major (d contiguous): k step kk = page kk = [2 halves][16 tok][128 B];
+              // 2 KB between the two 64-column halves, 1 KB between its two 8-token groups
+              const uint64_t bd = smem_desc(v_base + kk * kPageBytes, kPageHalf, 1024);
               umma(tmem + 384, ad, bd, kIdescPV, (kk > 0) || !fresh);
             }
             umma_commit(bar(B_O_FULL + b));
@@ -380,6 +428,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
             for (int kk = 0; kk < kD / 16; ++kk) {
               const uint64_t ad = smem_desc(q_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
+              // B = K [2 halves][128 tok][128 B], K-major: 8-token groups 1 KB apart
               const uint64_t bd = smem_desc(k_base + (kk >> 2) * kHalfSlot + (kk & 3) * 32, 16, 1024);
               umma(tmem + b3 * 128, ad, bd, kIdescS, kk > 0);
             }
@@ -392,6 +441,9 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
             progressed = true;
           }
         }
+#ifdef DSCALE_TRACE
+        ++mma_loops; if (!progressed) ++mma_idle;
+#endif
         if (progressed) {
           t_idle = clock64();
         } else {
@@ -399,9 +451,13 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           else if (clock64() - t_idle > kWaitCycles) { *s_abort = 1; ok = false; }
         }
       }
+#ifdef DSCALE_TRACE
+      { unsigned long long* trp = ws_ptr<unsigned long long>(a.ws, L.trace) + (size_t)c * 64;
+        trp[42] = mma_loops; trp[43] = mma_idle; trp[44] = clock64() - mma_t0; }
+#endif
     }
     __syncwarp();
-  } else if (warp == 6) {
+  } else if (warp == kWarpPublisher) {
     // ========================================================= publisher warp
     // Publishes the partial of the slice's first run in the background: waits
     // until the softmax threads have stored it, fences, and takes a ticket on the
@@ -414,7 +470,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         __threadfence();
         if (lane == 0) {
           const long long p0 = ((long long)s_tile[sg.i] * n_kv) + (long long)sg.g * sg.n_tiles;
-          const int n_contrib = cta_of(p0 + sg.n_tiles - 1, T, C) - cta_of(p0, T, C) + 1;
+          const int n_contrib = cta_of(p0 + sg.n_tiles - 1) - cta_of(p0) + 1;
           int* cnt = &ws_ptr<int>(a.ws, L.pair_cnt)[sg.i * n_kv + sg.g];
           const int old = atomicAdd(cnt, 1);
           *s_head_last = (old == n_contrib - 1);          // then this CTA merges it after its loop
@@ -425,7 +481,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     }
     __syncwarp();
   } else {
-    // ====================================================== softmax warps 0-3
+    // ====================================================== softmax warps 0-7
     // rows of capacity beyond M_live are written as zero, spread over the grid
     {
       const int m_live = hdr[H_M_LIVE];
@@ -436,13 +492,16 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
            x += (long long)gridDim.x * kSoftmaxThreads)
         dst[x] = make_uint4(0, 0, 0, 0);
     }
-    // Thread t of warp w works on two tile rows, rA = 16 w + t / 4 and rB = rA + 8
-    // (tile row m = 4 j + h_local), and on the column pairs 8 n + 2 (t % 4) + {0, 1},
-    // n = 0..15: the layout tcgen05.ld.16x256b gives, so all 32 lanes carry 64 of
-    // the warp's 16 x 128 scores.  A row is shared by the 4 threads of a quad.
+    // Warp w reads the TMEM lanes of q-head wq = w % 4 (tile rows 16 wq .. 16 wq + 15) and
+    // works on window rows j = 8 (w / 4) + 0..7 of it.  tcgen05.ld.16x256b hands thread t,
+    // for each 8-column group n, the column pair 8 n + 2 (t % 4) + {0, 1} of row t / 4 and
+    // of row t / 4 + 8; the thread keeps the pair of its own row.  A row is shared by the
+    // 4 threads of a quad.
     const int quad = lane & 3;
-    const int rowv[2] = {warp * 16 + (lane >> 2), warp * 16 + (lane >> 2) + 8};
-    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    const int wq = warp & 3, half = warp >> 2;
+    const int j_row = 8 * half + (lane >> 2);          // window slot of this thread's row
+    const int m_row = 16 * wq + j_row;                 // its tile row
+    const uint32_t t_lane = tmem + ((uint32_t)(wq * 32) << 16);
     const uint32_t o_addr = t_lane + 384;
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
     float* part_o = ws_ptr<float>(a.ws, L.part_o);
@@ -474,45 +533,51 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       v += __shfl_xor_sync(0xffffffffu, v, 1);
       return v + __shfl_xor_sync(0xffffffffu, v, 2);
     };
+    // this thread's 32 values (16 column pairs) of a 16-lane x 128-column TMEM block
+    auto load_own = [&](uint32_t taddr, float* v) {
+      float r[64];
+      tmem_ld_16x128(taddr, r);
+#pragma unroll
+      for (int n = 0; n < 16; ++n) {
+        v[2 * n] = half ? r[4 * n + 2] : r[4 * n];
+        v[2 * n + 1] = half ? r[4 * n + 3] : r[4 * n + 1];
+      }
+    };
     // fold a partial (O row in shared memory at o_row, its (max, sum) = ml) into this
-    // thread's share of row h of acc
-    auto fold_row = [&](float* acc, int h, float& m_run, float& l_run, uint32_t o_row, float2 ml) {
+    // thread's share of its row
+    auto fold_row = [&](float* acc, float& m_run, float& l_run, uint32_t o_row, float2 ml) {
       const float m_tot = fmaxf(m_run, ml.x);
       const float m_s = (m_tot == -INFINITY) ? 0.0f : m_tot;
       const float w_me = ex2(m_run - m_s), w_o = ex2(ml.x - m_s);
 #pragma unroll
       for (int n = 0; n < 16; ++n) {
         const float2 v = ld_shared_v2f(o_row + (8 * n + 2 * quad) * 4);
-        acc[4 * n + 2 * h] = acc[4 * n + 2 * h] * w_me + v.x * w_o;
-        acc[4 * n + 2 * h + 1] = acc[4 * n + 2 * h + 1] * w_me + v.y * w_o;
+        acc[2 * n] = acc[2 * n] * w_me + v.x * w_o;
+        acc[2 * n + 1] = acc[2 * n + 1] * w_me + v.y * w_o;
       }
       l_run = l_run * w_me + ml.y * w_o;
       m_run = m_tot;
     };
-    // normalise and write this thread's share of row h: 16 column pairs
-    auto write_row = [&](const float* acc, int h, float l, int oi, int g) {
+    // normalise and write this thread's share of its row: 16 column pairs
+    auto write_row = [&](const float* acc, float l, int oi, int g) {
       const float inv = 1.0f / l;
-      __nv_bfloat16* dst = out + ((size_t)(oi + (rowv[h] >> 2)) * Hq + g * 4 + (rowv[h] & 3)) * kD + 2 * quad;
+      __nv_bfloat16* dst = out + ((size_t)(oi + j_row) * Hq + g * 4 + wq) * kD + 2 * quad;
 #pragma unroll
       for (int n = 0; n < 16; ++n)
-        *reinterpret_cast<uint32_t*>(dst + 8 * n) = pack_bf16(acc[4 * n + 2 * h] * inv, acc[4 * n + 2 * h + 1] * inv);
+        *reinterpret_cast<uint32_t*>(dst + 8 * n) = pack_bf16(acc[2 * n] * inv, acc[2 * n + 1] * inv);
     };
 
     while (ok && sch.next(sg)) {
       const int ki = ws_ptr<int>(a.ws, L.k)[sg.i];
       const int oi = ws_ptr<int>(a.ws, L.offset)[sg.i];
       const int len = kv_len[sg.i];
-      bool live[2];
-      int pos[2];
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        live[h] = (rowv[h] >> 2) < ki;
-        pos[h] = live[h] ? ws_ptr<int>(a.ws, L.positions)[oi + (rowv[h] >> 2)] : -1;
-      }
+      const bool live = j_row < ki;
+      const bool warp_live = 8 * half < ki;            // warp-uniform: some row of this warp is live
+      const int pos = live ? ws_ptr<int>(a.ws, L.positions)[oi + j_row] : -1;
       // O accumulates in TMEM relative to a reference maximum m_ref that is only
       // raised (and O rescaled) when the row maximum outgrows it by 2^8.  l_part
       // is this thread's share of the row sum (summed over the quad at the end).
-      float m_ref[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.0f, 0.0f};
+      float m_ref = -INFINITY, l_part = 0.0f;
 
       for (int t = sg.t0; t < sg.t1 && ok; ++t, ++it) {
         const int b = it & 1;
@@ -523,103 +588,115 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         ok = mbar_wait(bar(B_S_FULL + b3), (it / 3) & 1, s_abort);
         if (!ok) break;
         tc_fence_after();
+        // A warp without live rows only keeps in step: its arrival on the P barrier of tile
+        // `it` must not land in the phase of tile it - 2, which ends with that tile's P.V.
+        if (!warp_live && it >= 2) { ok = wait_pv(it - 2); if (!ok) break; }
 #ifdef DSCALE_TRACE
         if (t == sg.t0) { TRACE(tr); ++tr; }
         const long long tw1 = clock64();
         wait_cycles += tw1 - tw0;
 #endif
-        float s[64];
-        tmem_ld_16x128(t_lane + b3 * 128, s);
+        if (warp_live) {
+          float s[32];
+          load_own(t_lane + b3 * 128, s);
 #ifdef DSCALE_TRACE
-        const long long tw2 = clock64();
-        c_ld += tw2 - tw1;
+          const long long tw2 = clock64();
+          c_ld += tw2 - tw1;
 #endif
-        int vis[2];
-        float mx[2];
-        bool need = false;
-        float factor[2] = {1.0f, 1.0f};
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          vis[h] = min(kTileTok, max(0, pos[h] + 1 - t * kTileTok));     // visible columns of the row
+          const int vis = min(kTileTok, max(0, pos + 1 - t * kTileTok));     // visible columns of the row
           float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-          if (vis[h] >= kTileTok) {
+          if (vis >= kTileTok) {
 #pragma unroll
             for (int n = 0; n < 16; ++n) {
-              m4[(2 * n) & 3] = fmaxf(m4[(2 * n) & 3], s[4 * n + 2 * h]);
-              m4[(2 * n + 1) & 3] = fmaxf(m4[(2 * n + 1) & 3], s[4 * n + 2 * h + 1]);
+              m4[(2 * n) & 3] = fmaxf(m4[(2 * n) & 3], s[2 * n]);
+              m4[(2 * n + 1) & 3] = fmaxf(m4[(2 * n + 1) & 3], s[2 * n + 1]);
             }
           } else {
 #pragma unroll
             for (int n = 0; n < 16; ++n) {
               const int col = 8 * n + 2 * quad;
-              if (col < vis[h]) m4[(2 * n) & 3] = fmaxf(m4[(2 * n) & 3], s[4 * n + 2 * h]);
-              if (col + 1 < vis[h]) m4[(2 * n + 1) & 3] = fmaxf(m4[(2 * n + 1) & 3], s[4 * n + 2 * h + 1]);
+              if (col < vis) m4[(2 * n) & 3] = fmaxf(m4[(2 * n) & 3], s[2 * n]);
+              if (col + 1 < vis) m4[(2 * n + 1) & 3] = fmaxf(m4[(2 * n + 1) & 3], s[2 * n + 1]);
             }
           }
-          mx[h] = quad_max(fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]))) * scale_log2;
+          const float mx = quad_max(fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]))) * scale_log2;
+          bool need = false;
+          float factor = 1.0f;
           if (t == sg.t0) {
-            m_ref[h] = mx[h];                          // the run's first P.V starts a fresh O
-          } else if (live[h] && mx[h] > m_ref[h] + 8.0f) {
-            factor[h] = ex2(m_ref[h] - mx[h]);
-            m_ref[h] = mx[h];
-            l_part[h] *= factor[h];
+            m_ref = mx;                                // the run's first P.V starts a fresh O
+          } else if (live && mx > m_ref + 8.0f) {
+            factor = ex2(m_ref - mx);
+            m_ref = mx;
+            l_part *= factor;
             need = true;
           }
-        }
-        if (__any_sync(0xffffffffu, need)) {
-          // rescale this warp's O rows in TMEM before the next P.V accumulates
-          ok = wait_pv(it - 1);
-          if (!ok) break;
-          tc_fence_after();
-          float o[64];
-          tmem_ld_16x128(o_addr, o);
+          if (__any_sync(0xffffffffu, need)) {
+            // Rescale this warp's O rows in TMEM before the next P.V accumulates.  The
+            // 16-lane load / store also carries the sibling warp's 8 rows (written back
+            // unchanged), so the two warps of a q-head take turns.
+            ok = wait_pv(it - 1);
+            if (!ok) break;
+            if (lane == 0) {
+              const long long t0 = clock64();
+              while (atomicCAS(const_cast<int*>(&s_lock[wq]), 0, 1) != 0) {
+                if (*s_abort || clock64() - t0 > kWaitCycles) { *s_abort = 1; break; }
+              }
+            }
+            __syncwarp();
+            if (*s_abort) { ok = false; break; }
+            tc_fence_after();
+            float o[64];
+            tmem_ld_16x128(o_addr, o);
 #pragma unroll
-          for (int n = 0; n < 16; ++n) {
-            o[4 * n] *= factor[0]; o[4 * n + 1] *= factor[0];
-            o[4 * n + 2] *= factor[1]; o[4 * n + 3] *= factor[1];
+            for (int n = 0; n < 16; ++n) {
+              if (half) { o[4 * n + 2] *= factor; o[4 * n + 3] *= factor; }
+              else { o[4 * n] *= factor; o[4 * n + 1] *= factor; }
+            }
+            tmem_st_16x128(o_addr, o);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { __threadfence_block(); atomicExch(const_cast<int*>(&s_lock[wq]), 0); }
           }
-          tmem_st_16x128(o_addr, o);
-          tmem_st_wait();
-        }
 #ifdef DSCALE_TRACE
-        const long long tw3 = clock64();
-        c_max += tw3 - tw2;
+          const long long tw3 = clock64();
+          c_max += tw3 - tw2;
 #endif
-        // P[b] was last read by the P.V of tile it - 2
-        if (it >= 2) { ok = wait_pv(it - 2); if (!ok) break; }
+          // P[b] was last read by the P.V of tile it - 2
+          if (it >= 2) { ok = wait_pv(it - 2); if (!ok) break; }
 #ifdef DSCALE_TRACE
-        const long long tw4 = clock64();
-        c_pvw += tw4 - tw3;
+          const long long tw4 = clock64();
+          c_pvw += tw4 - tw3;
 #endif
-        const uint32_t p_base = base + kOffP + b * kPBytes + quad * 4;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const float m_safe = (m_ref[h] == -INFINITY) ? 0.0f : m_ref[h];
-          const uint32_t p_row = p_base + rowv[h] * 128;
-          const int sw = rowv[h] & 7;
+          const float m_safe = (m_ref == -INFINITY) ? 0.0f : m_ref;
+          const uint32_t p_row = base + kOffP + b * kPBytes + quad * 4 + m_row * 128;
+          const int sw = m_row & 7;
           float ps0 = 0.0f, ps1 = 0.0f;
-          if (vis[h] >= kTileTok) {
+          if (vis >= kTileTok) {
             // every column visible (all tiles but a pair's last one or two)
 #pragma unroll
             for (int n = 0; n < 16; ++n) {
-              const float p0 = ex2(fmaf(s[4 * n + 2 * h], scale_log2, -m_safe));
-              const float p1 = ex2(fmaf(s[4 * n + 2 * h + 1], scale_log2, -m_safe));
+              const float p0 = ex2(fmaf(s[2 * n], scale_log2, -m_safe));
+              const float p1 = ex2(fmaf(s[2 * n + 1], scale_log2, -m_safe));
               ps0 += p0; ps1 += p1;
               st_shared_b32(p_row + (n >> 3) * (kTcRows * 128) + (((n & 7) ^ sw) << 4), pack_bf16(p0, p1));
             }
-          } else if (live[h]) {
+          } else if (live) {
 #pragma unroll
             for (int n = 0; n < 16; ++n) {
               const int col = 8 * n + 2 * quad;
-              float p0 = ex2(fmaf(s[4 * n + 2 * h], scale_log2, -m_safe));
-              float p1 = ex2(fmaf(s[4 * n + 2 * h + 1], scale_log2, -m_safe));
-              p0 = (col < vis[h]) ? p0 : 0.0f;
-              p1 = (col + 1 < vis[h]) ? p1 : 0.0f;
+              float p0 = ex2(fmaf(s[2 * n], scale_log2, -m_safe));
+              float p1 = ex2(fmaf(s[2 * n + 1], scale_log2, -m_safe));
+              p0 = (col < vis) ? p0 : 0.0f;
+              p1 = (col + 1 < vis) ? p1 : 0.0f;
               ps0 += p0; ps1 += p1;
               st_shared_b32(p_row + (n >> 3) * (kTcRows * 128) + (((n & 7) ^ sw) << 4), pack_bf16(p0, p1));
             }
           }
-          l_part[h] += ps0 + ps1;
+          l_part += ps0 + ps1;
+#ifdef DSCALE_TRACE
+          c_exp += clock64() - tw4;
+#endif
         }
         // last tile of the pair: V rows at or beyond the request's key count
         // must be finite (0 x NaN would poison the row): zero them once the
@@ -634,12 +711,11 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           const uint32_t v_base = base + kOffKV + slot * kSlotBytes;
           for (int x = tid; x < n_chunks; x += kSoftmaxThreads) {
             const int r = first + (x >> 4), hc = x & 15;
-            st_shared_v4(v_base + (hc >> 3) * kHalfSlot + r * 128 + ((hc & 7) << 4), 0, 0, 0, 0);
+            st_shared_v4(v_base + (r >> 4) * kPageBytes + (hc >> 3) * kPageHalf + (r & 15) * 128 + ((hc & 7) << 4), 0, 0, 0, 0);
           }
         }
 #ifdef DSCALE_TRACE
         const long long tw5 = clock64();
-        c_exp += tw5 - tw4;
 #endif
         tc_fence_before();
         fence_async_smem();
@@ -659,10 +735,10 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       TRACE(tr); ++tr;
 #endif
       tc_fence_after();
-      float acc[64];
-      tmem_ld_16x128(o_addr, acc);
+      float acc[32];
+      load_own(o_addr, acc);
       tc_fence_before();
-      float l_run[2] = {quad_sum(l_part[0]), quad_sum(l_part[1])};
+      float l_run = quad_sum(l_part);
 
       const int kind = run_kind(sg, sch.more());
       bool write_rows = (kind == RUN_WHOLE);
@@ -673,16 +749,13 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         const int fast = *s_fast;
         if (fast > 0) {
           // all other contributors' partials sit in ring slots 2 it, 2 it + 1, ...:
-          // fold them into this thread's rows and finish the pair here
+          // fold them into this thread's row and finish the pair here
           const uint32_t ml_base = base + kOffQ + ((seg + 1) & 1) * kQBytes;
           for (int x = 0; x < fast; ++x) {
             const uint32_t o_slot = base + kOffKV + ((2 * it + x) % kStages) * kSlotBytes;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              if (live[h])
-                fold_row(acc, h, m_ref[h], l_run[h], o_slot + rowv[h] * (kD * 4),
-                         ld_shared_v2f(ml_base + (x * kTcRows + rowv[h]) * 8));
-            }
+            if (live)
+              fold_row(acc, m_ref, l_run, o_slot + m_row * (kD * 4),
+                       ld_shared_v2f(ml_base + (x * kTcRows + m_row) * 8));
           }
           if (tid == 0) pair_cnt[sg.i * n_kv + sg.g] = 0;      // ready for the next launch
           write_rows = true;
@@ -690,27 +763,20 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           store_partial = true;                                // ordinary path after the loop
         }
       }
-      if (write_rows) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-          if (live[h]) write_row(acc, h, l_run[h], oi, sg.g);
-      }
+      if (write_rows && live) write_row(acc, l_run, oi, sg.g);
       if (store_partial) {
         // A run that covers only part of its pair: store the un-normalised partial.
         // Nothing in the main loop waits on global memory (a round trip costs
         // microseconds while every SM is streaming).
         const int slot_id = c * 2 + (sg.first_of_cta ? 0 : 1);
+        if (live) {
+          float* po = part_o + ((size_t)slot_id * kTcRows + m_row) * kD + 2 * quad;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (live[h]) {
-            float* po = part_o + ((size_t)slot_id * kTcRows + rowv[h]) * kD + 2 * quad;
-#pragma unroll
-            for (int n = 0; n < 16; ++n)
-              *reinterpret_cast<float2*>(po + 8 * n) = make_float2(acc[4 * n + 2 * h], acc[4 * n + 2 * h + 1]);
-            if (quad == 0)
-              *reinterpret_cast<float2*>(&part_ml[((size_t)slot_id * kTcRows + rowv[h]) * 2]) =
-                  make_float2(m_ref[h], l_run[h]);
-          }
+          for (int n = 0; n < 16; ++n)
+            *reinterpret_cast<float2*>(po + 8 * n) = make_float2(acc[2 * n], acc[2 * n + 1]);
+          if (quad == 0)
+            *reinterpret_cast<float2*>(&part_ml[((size_t)slot_id * kTcRows + m_row) * 2]) =
+                make_float2(m_ref, l_run);
         }
         if (kind == RUN_PUBLISH) {
           mbar_arrive(bar(B_PART));                            // the publisher warp takes over
@@ -733,7 +799,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     // ---- end phase: publish what is left, merge the pairs this CTA is last to reach
     if (ok && (fin_i >= 0 || head_i >= 0)) {
       unsigned group_phase = 0, merge_phase = 0;
-      auto group_sync = [&]() -> bool {                 // bounded barrier of the 128 softmax threads
+      auto group_sync = [&]() -> bool {                 // bounded barrier of the softmax threads
         mbar_arrive(bar(B_GROUP));
         const bool r = mbar_wait(bar(B_GROUP), group_phase & 1, s_abort);
         ++group_phase;
@@ -745,7 +811,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         ok = group_sync();
         if (ok && tid == 0) {
           const long long p0 = ((long long)s_tile[fin_i] * n_kv) + (long long)fin_g * fin_n;
-          const int n_contrib = cta_of(p0 + fin_n - 1, T, C) - cta_of(p0, T, C) + 1;
+          const int n_contrib = cta_of(p0 + fin_n - 1) - cta_of(p0) + 1;
           int* cnt = &pair_cnt[fin_i * n_kv + fin_g];
           const int old = atomicAdd(cnt, 1);
           s_ticket[0] = (old == n_contrib - 1);
@@ -759,19 +825,19 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         if (ok && *s_head_last) { merge_i[n_merge] = head_i; merge_g[n_merge] = head_g; merge_n[n_merge] = head_n; ++n_merge; }
       }
       // Merge: all contributors' partials are bulk-copied into the (now idle) K/V
-      // ring, up to kStages at a time, and every thread folds its share of its rows.
+      // ring, up to kStages at a time, and every thread folds its share of its row.
       for (int x = 0; ok && x < n_merge; ++x) {
         __threadfence();
         const int pi = merge_i[x], pg = merge_g[x];
         const int ki = ws_ptr<int>(a.ws, L.k)[pi];
         const int oi = ws_ptr<int>(a.ws, L.offset)[pi];
-        const bool live[2] = {(rowv[0] >> 2) < ki, (rowv[1] >> 2) < ki};
+        const bool live = j_row < ki;
         const long long p0 = ((long long)s_tile[pi] * n_kv) + (long long)pg * merge_n[x];
-        const int c_lo = cta_of(p0, T, C), c_hi = cta_of(p0 + merge_n[x] - 1, T, C);
-        float acc[64];
-        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
+        const int c_lo = cta_of(p0), c_hi = cta_of(p0 + merge_n[x] - 1);
+        float acc[32];
+        float m_run = -INFINITY, l_run = 0.0f;
 #pragma unroll
-        for (int d = 0; d < 64; ++d) acc[d] = 0.0f;
+        for (int d = 0; d < 32; ++d) acc[d] = 0.0f;
         for (int cb = c_lo; cb <= c_hi && ok; cb += kStages) {
           const int nb = min(kStages, c_hi - cb + 1);
           ok = group_sync();                            // everybody is done with the ring slots
@@ -781,40 +847,29 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
             mbar_expect_tx(bar(B_MERGE), nb * kTcRows * kD * 4);
             for (int y = 0; y < nb; ++y) {
               const int cc = cb + y;
-              const int sid = cc * 2 + (slice_begin(cc, T, C) >= p0 ? 0 : 1);
+              const int sid = cc * 2 + (s_slice[cc] >= p0 ? 0 : 1);
               bulk_load(base + kOffKV + y * kSlotBytes, part_o + (size_t)sid * kTcRows * kD,
                         kTcRows * kD * 4, bar(B_MERGE));
             }
           }
-          float2 ml[kStages][2];
+          float2 ml[kStages];
 #pragma unroll
           for (int y = 0; y < kStages; ++y) {
             const int cc = min(cb + y, c_hi);
-            const int sid = cc * 2 + (slice_begin(cc, T, C) >= p0 ? 0 : 1);
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-              ml[y][h] = live[h] ? __ldcg(reinterpret_cast<const float2*>(&part_ml[((size_t)sid * kTcRows + rowv[h]) * 2]))
-                                 : make_float2(-INFINITY, 0.0f);
+            const int sid = cc * 2 + (s_slice[cc] >= p0 ? 0 : 1);
+            ml[y] = live ? __ldcg(reinterpret_cast<const float2*>(&part_ml[((size_t)sid * kTcRows + m_row) * 2]))
+                         : make_float2(-INFINITY, 0.0f);
           }
           ok = mbar_wait(bar(B_MERGE), merge_phase & 1, s_abort);
           ++merge_phase;
           if (!ok) break;
 #pragma unroll
           for (int y = 0; y < kStages; ++y) {
-            if (y < nb) {
-#pragma unroll
-              for (int h = 0; h < 2; ++h)
-                if (live[h])
-                  fold_row(acc, h, m_run[h], l_run[h],
-                           base + kOffKV + y * kSlotBytes + rowv[h] * (kD * 4), ml[y][h]);
-            }
+            if (y < nb && live)
+              fold_row(acc, m_run, l_run, base + kOffKV + y * kSlotBytes + m_row * (kD * 4), ml[y]);
           }
         }
-        if (ok) {
-#pragma unroll
-          for (int h = 0; h < 2; ++h)
-            if (live[h]) write_row(acc, h, l_run[h], oi, pg);
-        }
+        if (ok && live) write_row(acc, l_run, oi, pg);
       }
     }
   }
@@ -826,7 +881,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   tc_fence_before();
   __syncthreads();
   if (tid == 0 && *s_abort) atomicOr(&hdr[H_STATUS], 8 /*TIMEOUT*/);
-  if (warp == 5) {
+  if (warp == kWarpMma) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
   }
@@ -864,11 +919,16 @@ struct MapKey {
 std::mutex g_map_mu;
 std::map<MapKey, CUtensorMap> g_kv_maps, g_q_maps;
 
-// K or V of one layer: [num_pages][n_kv][16 tok][128 d] viewed as
-// (d_lo 64, d_hi 2, tok 16, head, page); one box = one page-head, 64 columns
-bool kv_map(const void* ptr, int n_kv, int num_pages, CUtensorMap* out) {
+// K or V of one layer: [num_pages][n_kv][16 tok][128 d].
+// whole_page = false (K): viewed as (d_lo 64, d_hi 2, tok 16, head, page), one box = one
+// 64-column half of a page-head, 2 KB, [16 tok][128 B]; the score product wants all 128
+// keys of a tile 128 bytes apart within a half.
+// whole_page = true (V): viewed as (d_lo 64, tok 16, d_hi 2, head, page), one box = one
+// whole page-head, 4 KB, landing as [2 column halves][16 tok][128 B]; the second product
+// takes one page per k step, so half the copy instructions do.
+bool kv_map(const void* ptr, int n_kv, int num_pages, bool whole_page, CUtensorMap* out) {
   std::lock_guard<std::mutex> lk(g_map_mu);
-  MapKey key{ptr, n_kv, num_pages};
+  MapKey key{ptr, n_kv, whole_page ? -num_pages : num_pages};
   auto it = g_kv_maps.find(key);
   if (it != g_kv_maps.end()) { *out = it->second; return true; }
   EncodeTiledFn enc = get_encode();
@@ -876,6 +936,11 @@ bool kv_map(const void* ptr, int n_kv, int num_pages, CUtensorMap* out) {
   cuuint64_t dims[5] = {64, 2, (cuuint64_t)kPage, (cuuint64_t)n_kv, (cuuint64_t)num_pages};
   cuuint64_t strides[4] = {128, 256, (cuuint64_t)kPage * kD * 2, (cuuint64_t)n_kv * kPage * kD * 2};
   cuuint32_t box[5] = {64, 1, (cuuint32_t)kPage, 1, 1};
+  if (whole_page) {
+    dims[1] = kPage; dims[2] = 2;
+    strides[0] = 256; strides[1] = 128;
+    box[1] = kPage; box[2] = 2;
+  }
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides,
                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -886,7 +951,8 @@ bool kv_map(const void* ptr, int n_kv, int num_pages, CUtensorMap* out) {
   return true;
 }
 
-// q: [rows][n_q][128] viewed as (d_lo 64, d_hi 2, head, row); box = 4 heads x 16 rows
+// q: [rows][n_q][128] viewed as (d_lo 64, d_hi 2, row, head); box = 16 rows x 4 heads, which
+// lands in shared memory head-major: tile row m = 16 h_local + j
 bool q_map(const void* ptr, int n_q, int rows, CUtensorMap* out) {
   std::lock_guard<std::mutex> lk(g_map_mu);
   MapKey key{ptr, n_q, rows};
@@ -894,9 +960,9 @@ bool q_map(const void* ptr, int n_q, int rows, CUtensorMap* out) {
   if (it != g_q_maps.end()) { *out = it->second; return true; }
   EncodeTiledFn enc = get_encode();
   if (!enc) return false;
-  cuuint64_t dims[4] = {64, 2, (cuuint64_t)n_q, (cuuint64_t)rows};
-  cuuint64_t strides[3] = {128, (cuuint64_t)kD * 2, (cuuint64_t)n_q * kD * 2};
-  cuuint32_t box[4] = {64, 1, 4, 16};
+  cuuint64_t dims[4] = {64, 2, (cuuint64_t)rows, (cuuint64_t)n_q};
+  cuuint64_t strides[3] = {128, (cuuint64_t)n_q * kD * 2, (cuuint64_t)kD * 2};
+  cuuint32_t box[4] = {64, 1, 16, 4};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides,
                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -921,11 +987,12 @@ cudaError_t attn_tc_prepare() {
 }
 
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t stream) {
+  if (a.num_ctas > kMaxCtas) return cudaErrorNotSupported;      // the slice table is staged in shared memory
   WsLayout L = ws_layout(a.n_bs, a.n_kv_heads, a.num_ctas);
   CUtensorMap tq, tk, tv;
   if (!q_map(a.q, a.n_q_heads, kHalfW * a.n_bs, &tq) ||
-      !kv_map(a.k_cache, a.n_kv_heads, a.num_pages, &tk) ||
-      !kv_map(a.v_cache, a.n_kv_heads, a.num_pages, &tv))
+      !kv_map(a.k_cache, a.n_kv_heads, a.num_pages, false, &tk) ||
+      !kv_map(a.v_cache, a.n_kv_heads, a.num_pages, true, &tv))
     return cudaErrorNotSupported;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(a.num_ctas);

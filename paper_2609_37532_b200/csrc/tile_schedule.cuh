@@ -78,6 +78,17 @@ __device__ __forceinline__ int cta_of(long long L, long long T, int C) {
   return (int)(((L + 1) * C + Tv - 1) / Tv) - 1;
 }
 
+// The packed kernel reads its slice starts from a table the allocation kernel writes
+// (equal-cost slices): tab[c] = first linear tile of CTA c, tab[C] = T, non-decreasing.
+// The CTA whose slice holds linear tile L: the last c with tab[c] <= L.
+__device__ __forceinline__ int cta_of_tab(const int* tab, int C, long long L) {
+  int lo = 0, hi = C;                      // invariant: tab[lo] <= L < tab[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (tab[mid] <= L) lo = mid; else hi = mid;
+  }
+  return lo;
+}
 
 }  // namespace
 }  // namespace dscale

@@ -19,6 +19,10 @@ constexpr int kMaxNbs = 64;
 constexpr int kTileTok = 128;     // keys per attention tile (8 pages)
 constexpr int kAccMaxChunks = 16; // vocab chunks per row in the argmax
 constexpr int kTcRows = 64;       // rows of the tensor-core query tile (GQA group 4 x 16 slots)
+// Cost of one key tile in the attention schedule, by the request's window length: with more
+// than 8 live rows per q-head the second group of softmax warps works too and a tile takes
+// about 4.5 % longer (measured).  Slices are cut to equal cost, not to equal tile counts.
+constexpr int kTileCostSmall = 64, kTileCostBig = 67;
 // acceptance-predictor front end ("Acceptance predictor" paragraph)
 constexpr int kPredPos = 15;          // new draft positions per request
 constexpr int kPredConf = 18;         // confidence values per position
@@ -39,7 +43,7 @@ enum HdrWord {
 struct WsLayout {
   size_t hdr, k, k0, offset, q_start, q_end, tokens, positions, kv_refs, row_req, top1,
       kv_len, tile_prefix, qscores, amax_val, amax_idx, smp_m, smp_s, row_m, row_z, row_flag, req_row, req_rej, pair_cnt, pad_cnt, lm_val, lm_idx,
-      part_o, part_ml, pred_part, pred_rowsum, pred_feat, trace, total;
+      part_o, part_ml, pred_part, pred_rowsum, pred_feat, slice_tab, trace, total;
 };
 
 __host__ __device__ inline size_t ws_align(size_t x) { return (x + 255) & ~size_t(255); }
@@ -89,6 +93,8 @@ __host__ __device__ inline WsLayout ws_layout(int n_bs, int n_kv_heads, int num_
   L.pred_part = o;   o = ws_align(o + size_t(kPredPos) * n_bs * kPredMaxChunks * kPredRec * 4);
   L.pred_rowsum = o; o = ws_align(o + size_t(kPredMaxChunks) * 32 * 4);
   L.pred_feat = o;   o = ws_align(o + size_t(n_bs) * kPredFeatures * 4);
+  // attention schedule: first linear key tile of every CTA's slice, [num_ctas + 1]
+  L.slice_tab = o;   o = ws_align(o + (size_t(num_ctas) + 1) * 4);
   // per-CTA timestamps, written only by builds with -DDSCALE_TRACE
   L.trace = o;       o = ws_align(o + size_t(num_ctas) * 64 * 8);
   L.total = o;

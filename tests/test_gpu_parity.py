@@ -217,6 +217,12 @@ def test_host_side_argument_validation(P):
     assert lib.dscale_alloc_verify(*bad) == -4
     bad = list(ok); bad[0] = C.c_void_p(ws.ptr + 256)   # not an initialised workspace
     assert lib.dscale_alloc_verify(*bad) == -4
+    # a destroyed workspace is unknown to every call until it is initialised again
+    assert lib.dscale_workspace_destroy(C.c_void_p(ws.ptr)) == 0
+    assert lib.dscale_workspace_destroy(C.c_void_p(ws.ptr)) == -4
+    assert lib.dscale_alloc_verify(*ok) == -4
+    assert lib.dscale_workspace_init(C.c_void_p(ws.ptr), ws.nbytes, 4, 8, 2, 128, ws.num_sms, null) == 0
+    assert lib.dscale_alloc_verify(*ok) == 0
     assert lib.dscale_workspace_bytes(65, 32, 8, 128, 148) == 0
     assert lib.dscale_workspace_bytes(8, 32, 8, 64, 148) == 0
     assert lib.dscale_workspace_bytes(8, 30, 8, 128, 148) == 0
