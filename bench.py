@@ -6,6 +6,9 @@
 One "step" is one pass of the whole hot path over one batch of seeded synthetic
 input, replayed as ONE captured CUDA graph.  The default workload is the
 Qwen3-8B-shaped full step at concurrency 32 (36 layers, contexts 2048-8192).
+Beside the headline (K replays between two barriers) the line carries the per-replay median and
+minimum, a sustained leg (seconds of replays, clock settled under the power cap), the attention
+kernel's roofline at both, the whole decision chain as one graph, and the CPU oracle's time.
 Prints one JSON line (rank 0).  With N > 1 (launched by torch.distributed.run)
 every rank runs an independent replica on its own GPU with its own batch:
 the path shards by request and needs no collective, so scaling is weak.
@@ -33,6 +36,8 @@ from dscale_inputs import (CONFIGS, make_kv_layer, make_lm_head_unpacked, make_l
 SCALE = 1.0 / float(np.sqrt(128.0))
 METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+FLUSH_BYTES = 384 * 1024 * 1024          # rewritten between replays of a step that fits the L2
 
 
 # --------------------------------------------------------------------- helpers
@@ -298,6 +303,26 @@ def run_ours(args, rank, world, local_rank):
             dist.barrier()
         torch.cuda.synchronize()
 
+    per_layer_b, per_step_b = algorithmic_bytes(cfg, req, k)
+    step_bytes = per_layer_b * cfg.layers + per_step_b
+    # A step whose inputs fit the 126 MB L2 is timed cold: a buffer larger than the L2 is
+    # rewritten before every replay (outside the per-replay events) and the step time is the
+    # sum of the per-replay intervals; the back-to-back (warm) figure is reported beside it.
+    flush = step_bytes < 4 * L2_BYTES
+    flush_buf = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev) if flush else None
+
+    def timed_replays(g, count, cold):
+        """Per-replay device times in ms (events on the launching stream)."""
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(2 * count)]
+        for s_ in range(count):
+            if cold:
+                flush_buf.fill_(s_ & 1)
+            evs[2 * s_].record(stream)
+            g.replay()
+            evs[2 * s_ + 1].record(stream)
+        barrier()
+        return np.array([evs[2 * s_].elapsed_time(evs[2 * s_ + 1]) for s_ in range(count)])
+
     sampler = ClockSampler(local_rank)
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
@@ -306,14 +331,24 @@ def run_ours(args, rank, world, local_rank):
         if rank == 0:
             sampler.start()
         # ---- timed region 1: K replays of the captured step (headline) ----
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
-        e0.record(stream)
-        for _ in range(args.steps):
-            graph.replay()
-        e1.record(stream)
-        barrier()
-        ms_total = e0.elapsed_time(e1)
+        if flush:
+            per_replay = timed_replays(graph, args.steps, cold=True)
+            ms_total = float(per_replay.sum())
+            warm_ms = float(np.median(timed_replays(graph, args.steps, cold=False)))
+        else:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+            e0.record(stream)
+            marks[0].record(stream)
+            for s_ in range(args.steps):
+                graph.replay()
+                marks[s_ + 1].record(stream)
+            e1.record(stream)
+            barrier()
+            ms_total = e0.elapsed_time(e1)
+            per_replay = np.array([marks[s_].elapsed_time(marks[s_ + 1]) for s_ in range(args.steps)])
+            warm_ms = None
 
         # ---- timed region 2: the dominant kernel alone, for its roofline: the L
         # attention launches of a step captured as their own graph (same launch
@@ -322,18 +357,10 @@ def run_ours(args, rank, world, local_rank):
         with torch.cuda.graph(g_attn, stream=stream):
             do_attn()
         g_attn.replay()
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-              for _ in range(args.steps)]
         barrier()
-        for s in range(args.steps):
-            ev[s][0].record(stream)
-            g_attn.replay()
-            ev[s][1].record(stream)
-        barrier()
-        _per = np.array([a.elapsed_time(b) for a, b in ev]) / max(1, cfg.layers)
-        if os.environ.get("DSCALE_BENCH_DEBUG"):
-            print("attn per-launch us by replay:", np.round(_per * 1e3, 1).tolist(), file=sys.stderr)
+        _per = timed_replays(g_attn, args.steps, cold=flush) / max(1, cfg.layers)
         attn_ms = float(np.mean(_per))
+        attn_med_ms, attn_min_ms = float(np.median(_per)), float(_per.min())
         ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ea.record(stream)
         for _ in range(args.steps):
@@ -410,6 +437,78 @@ def run_ours(args, rank, world, local_rank):
                     "frac_of_hbm_peak": pred_bytes / (pred_ms * 1e-3) / 1e9 / measured_peak()[0]}
             del pin
 
+        # ---- sustained legs: the same two graphs replayed for seconds, so that the clock has
+        # settled under the power cap; per-replay times over the last two thirds of the run
+        sustained = None
+        if args.sustain_s > 0 and not flush:
+            def sustained_leg(g, seconds, per_replay_ms):
+                smp = ClockSampler(local_rank)
+                count = max(20, int(seconds * 1e3 / per_replay_ms))
+                evs = [torch.cuda.Event(enable_timing=True) for _ in range(count + 1)]
+                barrier()
+                smp.start()
+                t_wall = time.perf_counter()
+                evs[0].record(stream)
+                for s_ in range(count):
+                    g.replay()
+                    evs[s_ + 1].record(stream)
+                barrier()
+                wall = time.perf_counter() - t_wall
+                clk = smp.stop()
+                per = np.array([evs[s_].elapsed_time(evs[s_ + 1]) for s_ in range(count)])
+                tail = per[count // 3:]
+                return {"replays": count, "wall_s": wall, "median_ms": float(np.median(tail)),
+                        "min_ms": float(tail.min()), "first_ms": float(np.median(per[:5])),
+                        "sm_mhz": clk.get("sm_mhz"), "reasons": clk.get("reasons")}
+            st_step = sustained_leg(graph, args.sustain_s, ms_total / args.steps)
+            st_attn = sustained_leg(g_attn, args.sustain_s * 2.0 / 3.0, attn_ms * cfg.layers)
+            sustained = {"step": st_step, "attn": st_attn}
+
+        # ---- the whole decision chain as one captured graph (Algorithm 2: features ->
+        # DVL, then target -> accept -> output): predictor front end -> allocation from its
+        # logits -> attention x L -> fused LM head + acceptance, on seeded drafter outputs
+        chain = None
+        if args.chain and args.lm_hidden > 0 and args.pred_hidden > 0 and args.attn == "tensor":
+            pin = make_predictor_inputs(req, args.pred_hidden, device=str(dev))
+            w_lm, h_un = make_lm_head_unpacked(req, args.lm_hidden, device=str(dev))
+            h_lm = rows_to_packed(h_un, k, offset, n, 8 * n_bs)
+            del h_un
+            pl_out = torch.zeros((n_bs, 15), dtype=torch.float32, device=dev)
+            co = [torch.zeros_like(x) for x in outs[:4]]
+
+            def chain_step():
+                P.predict_scores(ws, d_n_live, pin["draft_logits"], cfg.vocab, pin["draft_hidden"], pin["p_hidden"],
+                                 pin["p_logit"], pin["w1"], pin["b1"], pin["w2"], pin["b2"], pl_out)
+                P.alloc_verify(ws, d_n_live, pl_out, d_draft, d_ctx, d_bt, req["num_pages"], scores_are_logits=True)
+                do_attn()
+                P.lm_head_accept(ws, h_lm, w_lm, co[0], co[1], co[2], co[3])
+            chain_step()
+            barrier()
+            g_chain = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_chain, stream=stream):
+                chain_step()
+            for _ in range(3):
+                g_chain.replay()
+            barrier()
+            ch = timed_replays(g_chain, max(5, min(args.steps, 20)), cold=False)
+            k_chain = ws.field("k").cpu().numpy().copy()
+            kv_len = req["ctx_len"][:n].astype(np.int64) + k_chain[:n].astype(np.int64)
+            chain_bytes = (int(kv_len.sum()) * cfg.n_kv_heads * 128 * 2 * 2 + int(((kv_len + 15) // 16).sum()) * 4 +
+                           2 * 8 * n * cfg.n_q_heads * 128 * 2) * cfg.layers
+            chain_bytes += 15 * n * cfg.vocab * 4 + 32 * cfg.vocab * 2 + 15 * n * args.pred_hidden * 2     # drafter outputs
+            chain_bytes += w_lm.numel() * 2 + h_lm.numel() * 2                                              # LM head
+            ch_ms = float(np.median(ch))
+            chain = {"graph": "predict_scores -> alloc_verify (logits) -> verify_attn x %d -> lm_head_accept" % cfg.layers,
+                     "ms_per_step": ch_ms, "min_ms": float(ch.min()), "bytes": int(chain_bytes),
+                     "gbs": chain_bytes / (ch_ms * 1e-3) / 1e9,
+                     "frac_of_hbm_peak": chain_bytes / (ch_ms * 1e-3) / 1e9 / measured_peak()[0],
+                     "verified_tokens_per_step": int(co[3].sum().item()),
+                     "gpu_launches_per_step": P.lib.dscale_launches_per_call(7) + P.lib.dscale_launches_per_call(0) +
+                                              cfg.layers * P.lib.dscale_launches_per_call(1) + P.lib.dscale_launches_per_call(6)}
+            del pin, w_lm, h_lm, g_chain
+            do_alloc()                          # the workspace back to the canonical allocation
+            barrier()
+
         # ---- timed region 3: end to end through the host-buffer C ABI call ----
         hs = P.HostStep(ws, req["max_pages"], req["num_pages"], layers, logits, cfg.vocab, SCALE)
         hs.h_n_live[0] = n
@@ -438,7 +537,6 @@ def run_ours(args, rank, world, local_rank):
     e2e_value = e2e_tokens_all / e2e_s
 
     if rank == 0:
-        per_layer_b, per_step_b = algorithmic_bytes(cfg, req, k)
         peak, peak_kind = measured_peak()
         achieved = per_layer_b / (attn_ms * 1e-3) / 1e9
         step_gbs = (per_layer_b * cfg.layers + per_step_b) / (ms_step * 1e-3) / 1e9
@@ -449,10 +547,15 @@ def run_ours(args, rank, world, local_rank):
             "config": {"workload": cfg.name, "requests_per_gpu": n, "layers": cfg.layers,
                        "heads": [cfg.n_q_heads, cfg.n_kv_heads], "ctx": [cfg.ctx_lo, cfg.ctx_hi],
                        "vocab": cfg.vocab, "packed_rows": 8 * n, "attn": args.attn,
-                       "l2": "inputs_larger_than_L2 (%.1f GB per step)" %
-                             ((per_layer_b * cfg.layers + per_step_b) / 1e9),
+                       "l2": ("inputs_larger_than_L2 (%.1f GB per step)" % (step_bytes / 1e9)) if not flush else
+                             ("L2 flushed before every timed replay (a %d MB buffer rewritten; %.1f MB per step); "
+                              "step time = sum of the per-replay intervals" % (FLUSH_BYTES >> 20, step_bytes / 1e6)),
                        "launch": "one captured CUDA graph per step"},
             "verified_tokens_per_step": tokens_per_step,
+            "step_ms": {"mean": ms_step, "median": float(np.median(per_replay)), "min": float(per_replay.min()),
+                        "warm_median": warm_ms},
+            "sustained": sustained,
+            "decision_chain": chain,
             "packed_rows_per_s": 8 * n * world / (ms_step * 1e-3),
             "step_gbs": step_gbs, "step_frac_of_peak": step_gbs / peak,
             "step_frac_of_8tbs": step_gbs / 8000.0,
@@ -460,6 +563,10 @@ def run_ours(args, rank, world, local_rank):
                          "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                          "frac": achieved / peak, "frac_of_8tbs": achieved / 8000.0,
                          "bytes_per_launch": per_layer_b, "us_per_launch": attn_ms * 1e3,
+                         "us_per_launch_median": attn_med_ms * 1e3, "us_per_launch_min": attn_min_ms * 1e3,
+                         "frac_sustained": (per_layer_b / (sustained["attn"]["median_ms"] / cfg.layers * 1e-3) / 1e9 / peak)
+                                           if sustained else None,
+                         "us_per_launch_sustained": (sustained["attn"]["median_ms"] / cfg.layers * 1e3) if sustained else None,
                          "traffic": recorded_traffic(cfg.name)},
             "accept_us": accept_ms * 1e3, "accept_sampling_us": sampling_ms * 1e3,
             "lm_head_accept": lm, "predict_scores": pred,
@@ -503,6 +610,15 @@ def run_ours(args, rank, world, local_rank):
             v, work, desc = oracle_step_sample(cfg, req, kvs, qus, lu_cpu)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                     "sample": desc, "cpu_seconds": work}
+            try:                                 # the same oracle on one thread, on a smaller sample
+                from threadpoolctl import threadpool_limits
+                n_1 = max(1, min(2, n_l))
+                with threadpool_limits(limits=1):
+                    v1, work1, desc1 = oracle_step_sample(cfg, req, kvs[:n_1], qus[:n_1], lu_cpu)
+                line["cpu_baseline"]["single_thread"] = {"value": v1, "unit": UNIT, "cores": 1, "sample": desc1,
+                                                         "cpu_seconds": work1}
+            except Exception as e:               # threadpoolctl missing: say so, keep the threaded figure
+                line["cpu_baseline"]["single_thread"] = {"unavailable": str(e)}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -521,6 +637,10 @@ def main():
                     help="hidden size of the fused LM-head figure (0 skips it)")
     ap.add_argument("--pred-hidden", type=int, default=4096,
                     help="drafter hidden size of the predictor front-end figure (0 skips it)")
+    ap.add_argument("--sustain-s", type=float, default=3.0,
+                    help="seconds of back-to-back replays for the sustained legs (0 skips them)")
+    ap.add_argument("--no-chain", dest="chain", action="store_false",
+                    help="skip the full-size decision-chain graph (predictor -> allocation -> attention -> LM head)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-padded", action="store_true", help="skip the padded comparison kernel")
     ap.add_argument("--cpu-layers", type=int, default=0,

@@ -32,7 +32,7 @@
 //              clock drops under the power cap either count can bound the stream:
 //              24 copies and 16 products per tile keep both below the memory time
 //              (32 + 16 made the copies the bound, 16 + 24 the products).
-//   warp 9     one thread issues tcgen05.mma: S = Q K^T (M64 N128 K128, bf16 in,
+//   warp 9     issues tcgen05.mma (one lane; the warp's loop is warp-uniform): S = Q K^T (M64 N128 K128, bf16 in,
 //              fp32 in TMEM) for tile t, then O_t = P_{t-1} V_{t-1}; completion
 //              is signalled with tcgen05.commit on mbarriers.
 //   warps 0-7  softmax.  Tile rows are head-major (m = 16 h_local + j), so q-head
@@ -70,10 +70,7 @@ namespace {
 constexpr int kThreads = 352;
 constexpr int kSoftmaxThreads = 256;
 constexpr int kWarpProducer = 8, kWarpMma = 9, kWarpPublisher = 10;
-#ifndef DSCALE_STAGES
-#define DSCALE_STAGES 5
-#endif
-constexpr int kStages = DSCALE_STAGES;
+constexpr int kStages = 5;
 constexpr int kSlotBytes = kTileTok * kD * 2;           // 32 KB: one K or V tile
 constexpr int kHalfSlot = kSlotBytes / 2;               // K tile: one 64-column half [128 tok][128 B]
 constexpr int kPageBytes = kPage * kD * 2;              // V tile: 4 KB per page-head = one TMA box
@@ -112,14 +109,6 @@ constexpr uint32_t idesc(uint32_t n) {
 constexpr uint32_t kIdescS = idesc(128);
 constexpr uint32_t kIdescPV = idesc(128) | (1u << 16);
 
-#ifdef DSCALE_TRACE
-__device__ __forceinline__ unsigned long long gtime() {
-  unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t;
-}
-#define TRACE(slot) do { if (tid == 0 && (slot) < 64) trace[(slot)] = gtime(); } while (0)
-#else
-#define TRACE(slot) do { } while (0)
-#endif
 
 // How a run's result reaches the output.
 //   WHOLE    the run is its whole pair: rows are written directly.
@@ -158,9 +147,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int c = blockIdx.x;
-#ifdef DSCALE_TRACE
-  const unsigned long long t_entry = gtime();
-#endif
   int* hdr = ws_ptr<int>(a.ws, L.hdr);
   const int n_bs = a.n_bs, n_kv = a.n_kv_heads, Hq = a.n_q_heads;
 
@@ -214,8 +200,14 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   // with fewer tiles than CTAs only the first T CTAs get a (one-tile) slice, so
   // that every CTA in [0, C) has work and the per-pair contributor count is exact
   const int C = (int)min((long long)gridDim.x, T);
-  const long long sl_begin = c < C ? s_slice[c] : 0;
-  const long long sl_end = c < C ? s_slice[c + 1] : 0;
+  long long sl_begin = c < C ? s_slice[c] : 0;
+  long long sl_end = c < C ? s_slice[c + 1] : 0;
+  // a slice table that does not belong to this tile prefix (allocation not run on this
+  // workspace, or run for another grid) must not be followed
+  if (sl_begin < 0 || sl_begin > sl_end || sl_end > T || (c + 1 == C && sl_end != T)) {
+    if (tid == 0) atomicOr(&hdr[H_STATUS], 4 /*BAD_LEN*/);
+    sl_begin = sl_end = 0;
+  }
   auto cta_of = [&](long long Lt) { return cta_of_tab(s_slice, C, Lt); };
   const int* kv_len = ws_ptr<int>(a.ws, L.kv_len);
 
@@ -232,10 +224,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     const int pg_l = lane & 7, k_half = lane >> 3;
     // K/V are read exactly once per launch: mark them evict-first in L2
     const uint64_t kv_policy = make_policy_evict_first();
-#ifdef DSCALE_TRACE
-    long long prod_wait = 0, prod_fetch = 0;
-    const long long prod_t0 = clock64();
-#endif
     while (ok && sch.next(sg)) {
       const int qb = seg & 1;
       const int len = kv_len[sg.i];
@@ -255,13 +243,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
         for (int which = 0; which < 2; ++which, ++u) {
           const int slot = u % kStages;
-#ifdef DSCALE_TRACE
-          const long long pw0 = clock64();
-#endif
           if (!mbar_wait(bar(B_KV_EMPTY + slot), ((u / kStages) & 1) ^ 1, s_abort)) return false;
-#ifdef DSCALE_TRACE
-          prod_wait += clock64() - pw0;
-#endif
           if (lane == 0) mbar_expect_tx(bar(B_KV_FULL + slot), n_pages * kPageBytes);
           __syncwarp();
           if (which == 0) {
@@ -287,9 +269,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");
         waited = true;
-#ifdef DSCALE_TRACE
-        if (lane == 0) ws_ptr<unsigned long long>(a.ws, L.trace)[(size_t)c * 64 + 63] = gtime();
-#endif
         if (!ok) break;
       }
       ok = mbar_wait(bar(B_Q_EMPTY + qb), ((seg >> 1) & 1) ^ 1, s_abort);
@@ -303,13 +282,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       int page_next = t_first < sg.t1 ? fetch_page(t_first) : 0;
       for (int t = t_first; t < sg.t1 && ok; ++t) {
         const int page = page_next;
-#ifdef DSCALE_TRACE
-        const long long pf0 = clock64();
-#endif
         if (t + 1 < sg.t1) page_next = fetch_page(t + 1);
-#ifdef DSCALE_TRACE
-        prod_fetch += clock64() - pf0;
-#endif
         ok = issue_tile(t, page);
       }
       if (ok && run_kind(sg, sch.more()) == RUN_TAIL) {
@@ -351,10 +324,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       ++seg;
     }
     if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");
-#ifdef DSCALE_TRACE
-    if (lane == 0) { unsigned long long* trp = ws_ptr<unsigned long long>(a.ws, L.trace) + (size_t)c * 64;
-                     trp[40] = prod_wait; trp[41] = clock64() - prod_t0; trp[45] = prod_fetch; }
-#endif
     // on an aborted run, let the copies already issued land before the CTA's
     // shared memory is released (bounded, like every other wait)
     if (!ok) {
@@ -363,12 +332,20 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     }
   } else if (warp == kWarpMma) {
     // ============================================================ MMA issuer
-    if (lane == 0) {
-      // Event-driven issue.  S = Q K^T of tile x goes into TMEM buffer x % 3 as soon
-      // as its K slot has landed and that buffer's previous tile (x - 3) has been
-      // read by the softmax warps; O += P V of tile y as soon as P_y and V_y are
-      // there.  Scores may run up to two tiles ahead of the softmax, which frees K
-      // slots early and keeps more page copies in flight.
+    // Event-driven issue.  S = Q K^T of tile x goes into TMEM buffer x % 3 as soon
+    // as its K slot has landed and that buffer's previous tile (x - 3) has been
+    // read by the softmax warps; O += P V of tile y as soon as P_y and V_y are
+    // there.  Scores may run up to two tiles ahead of the softmax, which frees K
+    // slots early and keeps more page copies in flight.
+    // The whole warp runs the loop, so that cursors, barrier tests and descriptors are
+    // warp-uniform values; only the tcgen05 instructions themselves are issued by one
+    // lane.  Ring slots, phases and descriptors advance incrementally (no division, no
+    // descriptor rebuilt per instruction).
+    {
+      const bool leader = lane == 0;
+      auto ready = [&](uint32_t b_addr, uint32_t parity) {
+        return __all_sync(0xffffffffu, mbar_test(b_addr, parity));
+      };
       Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
       Segment sg;
       const unsigned total = (unsigned)(sl_end - sl_begin);
@@ -376,36 +353,42 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
       int seg = -1, t = 0, t_end = 0;            // S cursor: current run and tile inside it
       bool q_ready = false;
       unsigned run_start_mask = 0;               // bit (x % 4): tile x starts a run
+      // ring cursors: K of tile x is ring item 2 x, V is item 2 x + 1; item u sits in slot
+      // u % kStages in phase (u / kStages) & 1
+      int k_slot = 0, k_phase = 0, v_slot = 1 % kStages, v_phase = (1 / kStages) & 1;
+      int s_buf = 0;                             // score buffer next_s % 3
+      // descriptors of the operands at their base addresses; a k step adds a constant
+      const uint64_t q_desc0 = smem_desc(base + kOffQ, 16, 1024);
+      const uint64_t p_desc0 = smem_desc(base + kOffP, 16, 1024);
+      const uint64_t k_desc0 = smem_desc(base + kOffKV, 16, 1024);
+      const uint64_t v_desc0 = smem_desc(base + kOffKV, kPageHalf, 1024);
       bool ok = true;
       long long t_idle = clock64();
-#ifdef DSCALE_TRACE
-      long long mma_loops = 0, mma_idle = 0;
-      const long long mma_t0 = clock64();
-#endif
       while (ok && next_pv < total) {
         bool progressed = false;
         // ---- O += P V for the oldest tile whose P is ready
         if (next_pv < next_s) {
           const unsigned pt = next_pv;
           const int b = pt & 1;
-          const unsigned uv = 2 * pt + 1;
-          const int slot = uv % kStages;
-          if (mbar_test(bar(B_P_FULL + b), (pt >> 1) & 1) && mbar_test(bar(B_KV_FULL + slot), (uv / kStages) & 1)) {
+          if (ready(bar(B_P_FULL + b), (pt >> 1) & 1) && ready(bar(B_KV_FULL + v_slot), v_phase)) {
             tc_fence_after();
-            const uint32_t p_base = base + kOffP + b * kPBytes;
-            const uint32_t v_base = base + kOffKV + slot * kSlotBytes;
-            const bool fresh = (run_start_mask >> (pt & 3)) & 1;
+            // A = P [64 rows][128 tok] K-major: 64-token blocks of 8 KB, 32 B per 16 tokens.
+            // B = V, MN-major (d contiguous): k step kk = page kk = [2 halves][16 tok][128 B];
+            // 2 KB between the two 64-column halves, 1 KB between its two 8-token groups.
+            const uint64_t ad = p_desc0 + (uint64_t)(b * (kPBytes >> 4));
+            const uint64_t bd = v_desc0 + (uint64_t)(v_slot * (kSlotBytes >> 4));
+            const uint32_t fresh = (run_start_mask >> (pt & 3)) & 1;
+            if (leader) {
+              umma(tmem + 384, ad, bd, kIdescPV, fresh ^ 1u);
 #pragma unroll
-            for (int kk = 0; kk < kTileTok / 16; ++kk) {
-              // A = P [64 rows][128 tok] K-major: 64-token blocks of 8 KB, 32 B per 16 tokens
-              const uint64_t ad = smem_desc(p_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
-              // B = V, MN-major (d contiguous): k step kk = page kk = [2 halves][16 tok][128 B];
-              // 2 KB between the two 64-column halves, 1 KB between its two 8-token groups
-              const uint64_t bd = smem_desc(v_base + kk * kPageBytes, kPageHalf, 1024);
-              umma(tmem + 384, ad, bd, kIdescPV, (kk > 0) || !fresh);
+              for (int kk = 1; kk < kTileTok / 16; ++kk)
+                umma_acc(tmem + 384, ad + (uint64_t)((kk >> 2) * ((kTcRows * 128) >> 4) + (kk & 3) * 2),
+                         bd + (uint64_t)(kk * (kPageBytes >> 4)), kIdescPV);
+              umma_commit(bar(B_O_FULL + b));
+              umma_commit(bar(B_KV_EMPTY + v_slot));
             }
-            umma_commit(bar(B_O_FULL + b));
-            umma_commit(bar(B_KV_EMPTY + slot));
+            __syncwarp();
+            v_slot += 2; if (v_slot >= kStages) { v_slot -= kStages; v_phase ^= 1; }
             ++next_pv;
             progressed = true;
           }
@@ -417,33 +400,33 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
             ++seg; t = sg.t0; t_end = sg.t1; q_ready = false;
           }
           const int qb = seg & 1;
-          if (!q_ready) q_ready = mbar_test(bar(B_Q_FULL + qb), (seg >> 1) & 1);
-          const unsigned uk = 2 * next_s;
-          const int slot = uk % kStages;
-          if (q_ready && mbar_test(bar(B_KV_FULL + slot), (uk / kStages) & 1)) {
+          if (!q_ready) q_ready = ready(bar(B_Q_FULL + qb), (seg >> 1) & 1);
+          if (q_ready && ready(bar(B_KV_FULL + k_slot), k_phase)) {
             tc_fence_after();
-            const int b3 = next_s % 3;
-            const uint32_t q_base = base + kOffQ + qb * kQBytes;
-            const uint32_t k_base = base + kOffKV + slot * kSlotBytes;
+            // A = Q [64 rows][128 d], B = K [2 halves][128 tok][128 B], both K-major:
+            // 64-column blocks, 32 bytes per k step inside a block, 8-row groups 1 KB apart
+            const uint64_t ad = q_desc0 + (uint64_t)(qb * (kQBytes >> 4));
+            const uint64_t bd = k_desc0 + (uint64_t)(k_slot * (kSlotBytes >> 4));
+            const uint32_t d_s = tmem + s_buf * 128;
+            if (leader) {
+              umma_new(d_s, ad, bd, kIdescS);
 #pragma unroll
-            for (int kk = 0; kk < kD / 16; ++kk) {
-              const uint64_t ad = smem_desc(q_base + (kk >> 2) * (kTcRows * 128) + (kk & 3) * 32, 16, 1024);
-              // B = K [2 halves][128 tok][128 B], K-major: 8-token groups 1 KB apart
-              const uint64_t bd = smem_desc(k_base + (kk >> 2) * kHalfSlot + (kk & 3) * 32, 16, 1024);
-              umma(tmem + b3 * 128, ad, bd, kIdescS, kk > 0);
+              for (int kk = 1; kk < kD / 16; ++kk)
+                umma_acc(d_s, ad + (uint64_t)((kk >> 2) * ((kTcRows * 128) >> 4) + (kk & 3) * 2),
+                         bd + (uint64_t)((kk >> 2) * (kHalfSlot >> 4) + (kk & 3) * 2), kIdescS);
+              umma_commit(bar(B_S_FULL + s_buf));
+              umma_commit(bar(B_KV_EMPTY + k_slot));
+              if (t + 1 == t_end) umma_commit(bar(B_Q_EMPTY + qb));
             }
-            umma_commit(bar(B_S_FULL + b3));
-            umma_commit(bar(B_KV_EMPTY + slot));
-            if (t + 1 == t_end) umma_commit(bar(B_Q_EMPTY + qb));
+            __syncwarp();
             run_start_mask = (run_start_mask & ~(1u << (next_s & 3))) | ((t == sg.t0 ? 1u : 0u) << (next_s & 3));
+            k_slot += 2; if (k_slot >= kStages) { k_slot -= kStages; k_phase ^= 1; }
+            if (++s_buf == 3) s_buf = 0;
             ++t;
             ++next_s;
             progressed = true;
           }
         }
-#ifdef DSCALE_TRACE
-        ++mma_loops; if (!progressed) ++mma_idle;
-#endif
         if (progressed) {
           t_idle = clock64();
         } else {
@@ -451,10 +434,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           else if (clock64() - t_idle > kWaitCycles) { *s_abort = 1; ok = false; }
         }
       }
-#ifdef DSCALE_TRACE
-      { unsigned long long* trp = ws_ptr<unsigned long long>(a.ws, L.trace) + (size_t)c * 64;
-        trp[42] = mma_loops; trp[43] = mma_idle; trp[44] = clock64() - mma_t0; }
-#endif
     }
     __syncwarp();
   } else if (warp == kWarpPublisher) {
@@ -513,12 +492,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     Segment sg;
     unsigned it = 0;
     bool ok = true;
-#ifdef DSCALE_TRACE
-    unsigned long long* trace = ws_ptr<unsigned long long>(a.ws, L.trace) + (size_t)c * 64;
-    int tr = 2;
-    long long wait_cycles = 0, busy_cycles = 0, c_ld = 0, c_max = 0, c_pvw = 0, c_exp = 0, c_fence = 0;
-    if (tid == 0) { for (int x = 0; x < 64; ++x) trace[x] = 0; trace[0] = t_entry; trace[1] = gtime(); }
-#endif
     int head_i = -1, head_g = 0, head_n = 0;   // first run, published in the background
     int fin_i = -1, fin_g = 0, fin_n = 0;      // last run, published after the loop
     int seg = 0;
@@ -581,9 +554,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
 
       for (int t = sg.t0; t < sg.t1 && ok; ++t, ++it) {
         const int b = it & 1;
-#ifdef DSCALE_TRACE
-        const long long tw0 = clock64();
-#endif
         const int b3 = it % 3;                   // the three score buffers in TMEM
         ok = mbar_wait(bar(B_S_FULL + b3), (it / 3) & 1, s_abort);
         if (!ok) break;
@@ -591,18 +561,9 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         // A warp without live rows only keeps in step: its arrival on the P barrier of tile
         // `it` must not land in the phase of tile it - 2, which ends with that tile's P.V.
         if (!warp_live && it >= 2) { ok = wait_pv(it - 2); if (!ok) break; }
-#ifdef DSCALE_TRACE
-        if (t == sg.t0) { TRACE(tr); ++tr; }
-        const long long tw1 = clock64();
-        wait_cycles += tw1 - tw0;
-#endif
         if (warp_live) {
           float s[32];
           load_own(t_lane + b3 * 128, s);
-#ifdef DSCALE_TRACE
-          const long long tw2 = clock64();
-          c_ld += tw2 - tw1;
-#endif
           const int vis = min(kTileTok, max(0, pos + 1 - t * kTileTok));     // visible columns of the row
           float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
           if (vis >= kTileTok) {
@@ -658,16 +619,8 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
             __syncwarp();
             if (lane == 0) { __threadfence_block(); atomicExch(const_cast<int*>(&s_lock[wq]), 0); }
           }
-#ifdef DSCALE_TRACE
-          const long long tw3 = clock64();
-          c_max += tw3 - tw2;
-#endif
           // P[b] was last read by the P.V of tile it - 2
           if (it >= 2) { ok = wait_pv(it - 2); if (!ok) break; }
-#ifdef DSCALE_TRACE
-          const long long tw4 = clock64();
-          c_pvw += tw4 - tw3;
-#endif
           const float m_safe = (m_ref == -INFINITY) ? 0.0f : m_ref;
           const uint32_t p_row = base + kOffP + b * kPBytes + quad * 4 + m_row * 128;
           const int sw = m_row & 7;
@@ -694,9 +647,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
             }
           }
           l_part += ps0 + ps1;
-#ifdef DSCALE_TRACE
-          c_exp += clock64() - tw4;
-#endif
         }
         // last tile of the pair: V rows at or beyond the request's key count
         // must be finite (0 x NaN would poison the row): zero them once the
@@ -714,26 +664,13 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
             st_shared_v4(v_base + (r >> 4) * kPageBytes + (hc >> 3) * kPageHalf + (r & 15) * 128 + ((hc & 7) << 4), 0, 0, 0, 0);
           }
         }
-#ifdef DSCALE_TRACE
-        const long long tw5 = clock64();
-#endif
         tc_fence_before();
         fence_async_smem();
         mbar_arrive(bar(B_P_FULL + b));
-#ifdef DSCALE_TRACE
-        busy_cycles += clock64() - tw1;
-        c_fence += clock64() - tw5;
-#endif
       }
       if (!ok) break;
-#ifdef DSCALE_TRACE
-      TRACE(tr); ++tr;
-#endif
       ok = wait_pv(it - 1);                            // the run's last P.V
       if (!ok) break;
-#ifdef DSCALE_TRACE
-      TRACE(tr); ++tr;
-#endif
       tc_fence_after();
       float acc[32];
       load_own(o_addr, acc);
@@ -786,16 +723,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         }
       }
       ++seg;
-#ifdef DSCALE_TRACE
-      TRACE(tr); ++tr;
-#endif
     }
-#ifdef DSCALE_TRACE
-    TRACE(60);
-    if (tid == 0) { unsigned smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid)); trace[51] = smid;
-                    trace[58] = wait_cycles; trace[59] = busy_cycles; trace[57] = it;
-                    trace[52] = c_ld; trace[53] = c_max; trace[54] = c_pvw; trace[55] = c_exp; trace[56] = c_fence; }
-#endif
     // ---- end phase: publish what is left, merge the pairs this CTA is last to reach
     if (ok && (fin_i >= 0 || head_i >= 0)) {
       unsigned group_phase = 0, merge_phase = 0;
@@ -874,9 +802,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     }
   }
 
-#ifdef DSCALE_TRACE
-  if (tid == 0) ws_ptr<unsigned long long>(a.ws, L.trace)[(size_t)c * 64 + 61] = gtime();
-#endif
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
@@ -885,9 +810,6 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
   }
-#ifdef DSCALE_TRACE
-  if (tid == 0) ws_ptr<unsigned long long>(a.ws, L.trace)[(size_t)c * 64 + 62] = gtime();
-#endif
 }
 
 // ------------------------------------------------------------ host: tensor maps

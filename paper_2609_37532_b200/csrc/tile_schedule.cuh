@@ -50,11 +50,7 @@ struct Scheduler {
 // it would again finish last, launch after launch.  Three tiles and one tile less
 // (about 4.8 and 1.6 us of streaming) let them finish with the rest.
 __device__ __forceinline__ void slice_skew(long long T, int C, int& d1, int& d2) {
-#ifdef DSCALE_NO_SKEW
-  const bool on = false;
-#else
   const bool on = C >= 8 && T / C >= 24;
-#endif
   d1 = on ? 3 : 0;
   d2 = on ? 1 : 0;
 }

@@ -43,7 +43,7 @@ enum HdrWord {
 struct WsLayout {
   size_t hdr, k, k0, offset, q_start, q_end, tokens, positions, kv_refs, row_req, top1,
       kv_len, tile_prefix, qscores, amax_val, amax_idx, smp_m, smp_s, row_m, row_z, row_flag, req_row, req_rej, pair_cnt, pad_cnt, lm_val, lm_idx,
-      part_o, part_ml, pred_part, pred_rowsum, pred_feat, slice_tab, trace, total;
+      part_o, part_ml, pred_part, pred_rowsum, pred_feat, slice_tab, total;
 };
 
 __host__ __device__ inline size_t ws_align(size_t x) { return (x + 255) & ~size_t(255); }
@@ -95,8 +95,6 @@ __host__ __device__ inline WsLayout ws_layout(int n_bs, int n_kv_heads, int num_
   L.pred_feat = o;   o = ws_align(o + size_t(n_bs) * kPredFeatures * 4);
   // attention schedule: first linear key tile of every CTA's slice, [num_ctas + 1]
   L.slice_tab = o;   o = ws_align(o + (size_t(num_ctas) + 1) * 4);
-  // per-CTA timestamps, written only by builds with -DDSCALE_TRACE
-  L.trace = o;       o = ws_align(o + size_t(num_ctas) * 64 * 8);
   L.total = o;
   return L;
 }
