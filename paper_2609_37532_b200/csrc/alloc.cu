@@ -202,10 +202,13 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
     wreq[t] = -1;
   }
   // ---- attention schedule: slice c of the persistent grid starts at linear key tile
-  // slice_tab[c] (request-major, then kv-head, then tile).  Slices have equal cost; the
-  // last two CTAs of a launch, which start last, get three tiles and one tile less.
-  // Small tile counts (under 8 per CTA) are cut by count, and with fewer tiles than CTAs
-  // the first T CTAs get one tile each.
+  // slice_tab[c] (request-major, then kv-head, then tile).  Slices have equal COST under a
+  // measured model of the attention kernel: a tile of a request with more than 8 window rows
+  // costs 6 % more (both groups of softmax warps work), and every (request, kv-head) pair a
+  // CTA starts costs about 0.8 tile (epilogue of the previous pair, first scores of the next).
+  // The last CTAs of a launch start late (they land on the SMs that finished the previous
+  // launch last) and get two to three tiles less.  Small tile counts (under 8 per CTA) are
+  // cut by count, and with fewer tiles than CTAs the first T CTAs get one tile each.
   for (int cta = t; cta <= a.num_ctas; cta += blockDim.x) {
     const int n_kv = a.n_kv_heads;
     const long long T = (long long)sTilePre[kMaxNbs] * n_kv;
@@ -213,21 +216,35 @@ __global__ void __launch_bounds__(1024, 1) dvl_alloc_kernel(AllocArgs a, WsLayou
     long long tile = T;
     if (cta < C) {
       const bool by_count = T < 8 * C;
-      const bool skew = C >= 8 && T / C >= 24;
-      const int unit = by_count ? 1 : kTileCostSmall;
+      const int run_cost = by_count ? 0 : kRunCost;
+      auto tile_cost = [&](int r) { return by_count ? 1 : (sK[r] > 8 ? kTileCostBig : kTileCostSmall); };
       long long W = 0;
-      for (int r = 0; r < N; ++r) {
-        const int w = by_count ? 1 : (sK[r] > 8 ? kTileCostBig : kTileCostSmall);
-        W += (long long)(sTilePre[r + 1] - sTilePre[r]) * w * n_kv;
+      for (int r = 0; r < N; ++r)
+        W += ((long long)(sTilePre[r + 1] - sTilePre[r]) * tile_cost(r) + run_cost) * n_kv;
+      // late starters: the last kLateCtas CTAs give up kLateTiles[.] tiles each
+      const bool skew = !by_count && C >= 4 * kLateCtas && T / C >= 24;
+      long long pen_total = 0, pen_before = 0;
+      if (skew) {
+        for (int j = 0; j < kLateCtas; ++j) {
+          const long long pen = (long long)kLateTiles[j] * kTileCostSmall;
+          pen_total += pen;
+          if (C - kLateCtas + j < cta) pen_before += pen;
+        }
       }
-      const long long d1 = skew ? 3 * unit : 0, d2 = skew ? unit : 0;
-      const long long Wv = W + d1 + d2;                      // equal shares of a slightly longer list ...
-      const long long x = (cta == C - 1) ? (C - 1) * Wv / C - d2 : (long long)cta * Wv / C;   // ... the last two give some back
+      const long long Wv = W + pen_total;                    // equal shares of a slightly longer list ...
+      const long long x = (long long)cta * Wv / C - pen_before;   // ... of which the late starters give some back
       long long acc = 0;
       for (int r = 0; r < N; ++r) {
-        const int w = by_count ? 1 : (sK[r] > 8 ? kTileCostBig : kTileCostSmall);
-        const long long rc = (long long)(sTilePre[r + 1] - sTilePre[r]) * w * n_kv;
-        if (x < acc + rc) { tile = (long long)sTilePre[r] * n_kv + (x - acc) / w; break; }
+        const int n_r = sTilePre[r + 1] - sTilePre[r];
+        const long long pair_cost = (long long)n_r * tile_cost(r) + run_cost;
+        const long long rc = pair_cost * n_kv;
+        if (x < acc + rc) {
+          const long long g = (x - acc) / pair_cost, within = (x - acc) % pair_cost;
+          long long in_pair = within > run_cost ? (within - run_cost) / tile_cost(r) : 0;
+          if (in_pair >= n_r) in_pair = n_r - 1;
+          tile = (long long)sTilePre[r] * n_kv + g * n_r + in_pair;
+          break;
+        }
         acc += rc;
       }
     }

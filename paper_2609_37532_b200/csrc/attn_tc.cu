@@ -23,16 +23,17 @@
 // The grid and every address are independent of the lengths, so a captured
 // launch replays at any mix of lengths.
 //
-// Pipeline inside a CTA (352 threads):
-//   warp 8     producer: per tile, 16 TMA box copies of K (a 64-column half of one
+// Pipeline inside a CTA (32 (10 + kProducers) threads):
+//   warps 8..  producers (kProducers warps, each copying its share of every tile's pages):
+//              per tile, 16 TMA box copies of K (a 64-column half of one
 //              16-token page each, 2 KB) and 8 of V (a whole page-head, 4 KB), 128-byte
-//              swizzle, into a 5-deep ring of 32 KB slots; page ids are fetched one
-//              tile ahead.  Both the copy engine and the single MMA-issuing thread pay
+//              swizzle, into a 5-deep ring of 32 KB slots; page ids are fetched two
+//              tiles ahead.  Both the copy engine and the single MMA-issuing thread pay
 //              about 100 SM cycles per instruction whatever its size, and once the SM
 //              clock drops under the power cap either count can bound the stream:
 //              24 copies and 16 products per tile keep both below the memory time
 //              (32 + 16 made the copies the bound, 16 + 24 the products).
-//   warp 9     issues tcgen05.mma (one lane; the warp's loop is warp-uniform): S = Q K^T (M64 N128 K128, bf16 in,
+//   next warp  issues tcgen05.mma (one lane; the warp's loop is warp-uniform): S = Q K^T (M64 N128 K128, bf16 in,
 //              fp32 in TMEM) for tile t, then O_t = P_{t-1} V_{t-1}; completion
 //              is signalled with tcgen05.commit on mbarriers.
 //   warps 0-7  softmax.  Tile rows are head-major (m = 16 h_local + j), so q-head
@@ -46,7 +47,7 @@
 //              TMEM for a whole run of tiles (the second MMA accumulates onto
 //              it); it is only rescaled in place when a row maximum outgrows its
 //              reference by 2^8, and read back once per run for the epilogue.
-//   warp 10    publisher: fence + ticket for the first run's partial.
+//   last warp  publisher: fence + ticket for the first run's partial.
 // S is triple-buffered in TMEM (3 x 128 columns) next to O (128 columns), P and
 // Q are double-buffered in shared memory; the MMA thread issues whichever of the
 // two products is ready, scores up to two tiles ahead of the softmax.
@@ -67,9 +68,14 @@ namespace dscale {
 
 namespace {
 
-constexpr int kThreads = 352;
+#ifndef DSCALE_PRODUCERS
+#define DSCALE_PRODUCERS 2
+#endif
+constexpr int kProducers = DSCALE_PRODUCERS;            // copy-issuing warps (a power of two, at most 8)
+constexpr int kPagesPerProducer = (kTileTok / kPage) / kProducers;
 constexpr int kSoftmaxThreads = 256;
-constexpr int kWarpProducer = 8, kWarpMma = 9, kWarpPublisher = 10;
+constexpr int kWarpProducer = 8, kWarpMma = 8 + kProducers, kWarpPublisher = 9 + kProducers;
+constexpr int kThreads = 32 * (10 + kProducers);
 constexpr int kStages = 5;
 constexpr int kSlotBytes = kTileTok * kD * 2;           // 32 KB: one K or V tile
 constexpr int kHalfSlot = kSlotBytes / 2;               // K tile: one 64-column half [128 tok][128 B]
@@ -151,7 +157,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   const int n_bs = a.n_bs, n_kv = a.n_kv_heads, Hq = a.n_q_heads;
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(bar(B_KV_FULL + s), 1); mbar_init(bar(B_KV_EMPTY + s), 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(bar(B_KV_FULL + s), kProducers); mbar_init(bar(B_KV_EMPTY + s), 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar(B_Q_FULL + b), 1); mbar_init(bar(B_Q_EMPTY + b), 1);
       mbar_init(bar(B_P_FULL + b), kSoftmaxThreads);
@@ -194,7 +200,8 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
-  if (warp != kWarpProducer) asm volatile("griddepcontrol.wait;" ::: "memory");   // the producer waits later
+  const bool is_producer = warp >= kWarpProducer && warp < kWarpProducer + kProducers;
+  if (!is_producer) asm volatile("griddepcontrol.wait;" ::: "memory");   // the producers wait later
 
   const long long T = (long long)s_tile[n_bs] * n_kv;
   // with fewer tiles than CTAs only the first T CTAs get a (one-tile) slice, so
@@ -211,32 +218,43 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
   auto cta_of = [&](long long Lt) { return cta_of_tab(s_slice, C, Lt); };
   const int* kv_len = ws_ptr<int>(a.ws, L.kv_len);
 
-  if (warp == kWarpProducer) {
-    // ===================================================== TMA producer warp
+  if (is_producer) {
+    // ===================================================== TMA producer warps
+    // The copy engine takes about 50 cycles to accept an instruction from a single warp and
+    // then about one cycle per 43 bytes; instructions from several warps overlap the first
+    // part.  One warp alone cannot feed more than about 6 TB/s over the chip even from L2,
+    // so the boxes of a tile are spread over kProducers warps: warp pw copies pages
+    // pw * kPagesPerProducer .. of every K and V tile.  Only the first of them moves Q and
+    // the partner partials of the slice's last pair.
+    const int pw = warp - kWarpProducer;
     Scheduler sch; sch.init(s_tile, n_bs, n_kv, sl_begin, sl_end);
     Segment sg;
     unsigned u = 0;            // ring sequence number: K of tile it -> 2 it, V -> 2 it + 1
     int seg = 0;
     bool ok = true;
     bool waited = false;       // griddepcontrol.wait done
-    // V: lane l < 8 copies page l of the tile as one 4 KB box.  K: lanes l and l + 8 copy
-    // the two 64-column halves of page l as 2 KB boxes (see the shared-memory layouts below).
-    const int pg_l = lane & 7, k_half = lane >> 3;
+    // V: lane l < kPagesPerProducer copies one of this warp's pages as one 4 KB box.  K: lanes l
+    // and l + kPagesPerProducer copy the two 64-column halves of that page as 2 KB boxes.
+    const int pg_l = pw * kPagesPerProducer + (lane & (kPagesPerProducer - 1));
+    const int k_half = (lane / kPagesPerProducer) & 1;
     // K/V are read exactly once per launch: mark them evict-first in L2
     const uint64_t kv_policy = make_policy_evict_first();
     while (ok && sch.next(sg)) {
       const int qb = seg & 1;
       const int len = kv_len[sg.i];
       const int* bt = a.block_table + (size_t)sg.i * a.max_pages;
-      auto fetch_page = [&](int t) -> int {
+      // Page ids are loaded two tiles ahead and only looked at when their tile is issued: the
+      // load's round trip (several hundred cycles while every SM streams) then lies off this
+      // warp's path, which the copy instructions themselves already fill.
+      auto load_page = [&](int t) -> int {
         const int p = t * (kTileTok / kPage) + pg_l;
-        int id = 0;
-        if (lane < 16 && p * kPage < len) {
-          id = bt[p];
-          if (id < 0 || id >= a.num_pages) { atomicOr(&hdr[H_STATUS], 2); id = 0; }
-        }
+        return (lane < 2 * kPagesPerProducer && t < sg.t1 && p * kPage < len) ? __ldg(bt + p) : 0;
+      };
+      auto checked = [&](int id) -> int {
+        if (id < 0 || id >= a.num_pages) { atomicOr(&hdr[H_STATUS], 2); id = 0; }
         return id;
       };
+      auto fetch_page = [&](int t) -> int { return checked(load_page(t)); };
       auto issue_tile = [&](int t, int page) -> bool {       // K then V of key tile t into the ring
         const int valid_tok = min(kTileTok, len - t * kTileTok);
         const int n_pages = (valid_tok + kPage - 1) / kPage;
@@ -244,13 +262,14 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         for (int which = 0; which < 2; ++which, ++u) {
           const int slot = u % kStages;
           if (!mbar_wait(bar(B_KV_EMPTY + slot), ((u / kStages) & 1) ^ 1, s_abort)) return false;
-          if (lane == 0) mbar_expect_tx(bar(B_KV_FULL + slot), n_pages * kPageBytes);
+          const int mine = min(kPagesPerProducer, max(0, n_pages - pw * kPagesPerProducer));   // pages of this warp
+          if (lane == 0) mbar_expect_tx(bar(B_KV_FULL + slot), mine * kPageBytes);
           __syncwarp();
           if (which == 0) {
-            if (lane < 16 && pg_l < n_pages)
+            if (lane < 2 * kPagesPerProducer && pg_l < n_pages)
               tma_load_5d_hint(base + kOffKV + slot * kSlotBytes + k_half * kHalfSlot + pg_l * kPageHalf,
                                &tm_k, bar(B_KV_FULL + slot), 0, k_half, 0, sg.g, page, kv_policy);
-          } else if (lane < 8 && pg_l < n_pages) {
+          } else if (lane < kPagesPerProducer && pg_l < n_pages) {
             tma_load_5d_hint(base + kOffKV + slot * kSlotBytes + pg_l * kPageBytes,
                              &tm_v, bar(B_KV_FULL + slot), 0, 0, 0, sg.g, page, kv_policy);
           }
@@ -271,21 +290,22 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
         waited = true;
         if (!ok) break;
       }
-      ok = mbar_wait(bar(B_Q_EMPTY + qb), ((seg >> 1) & 1) ^ 1, s_abort);
+      if (pw == 0) ok = mbar_wait(bar(B_Q_EMPTY + qb), ((seg >> 1) & 1) ^ 1, s_abort);
       if (!ok) break;
-      if (lane == 0) {
+      if (pw == 0 && lane == 0) {
         mbar_expect_tx(bar(B_Q_FULL + qb), kQBytes);
         tma_load_4d(base + kOffQ + qb * kQBytes, &tm_q, bar(B_Q_FULL + qb), 0, 0, row0, sg.g * 4);
         tma_load_4d(base + kOffQ + qb * kQBytes + kQBytes / 2, &tm_q, bar(B_Q_FULL + qb), 0, 1,
                     row0, sg.g * 4);
       }
-      int page_next = t_first < sg.t1 ? fetch_page(t_first) : 0;
+      int page_1 = load_page(t_first), page_2 = load_page(t_first + 1);
       for (int t = t_first; t < sg.t1 && ok; ++t) {
-        const int page = page_next;
-        if (t + 1 < sg.t1) page_next = fetch_page(t + 1);
+        const int page = checked(page_1);
+        page_1 = page_2;
+        page_2 = load_page(t + 2);
         ok = issue_tile(t, page);
       }
-      if (ok && run_kind(sg, sch.more()) == RUN_TAIL) {
+      if (ok && pw == 0 && run_kind(sg, sch.more()) == RUN_TAIL) {
         // The slice ends inside this pair.  If every other contributor has already
         // published its partial (the usual case: they computed theirs at the start
         // of their slices), fetch those partials into ring slots behind the last
@@ -572,7 +592,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
               m4[(2 * n) & 3] = fmaxf(m4[(2 * n) & 3], s[2 * n]);
               m4[(2 * n + 1) & 3] = fmaxf(m4[(2 * n + 1) & 3], s[2 * n + 1]);
             }
-          } else {
+          } else if (vis > 0) {                        // (a row that is not live has vis = 0)
 #pragma unroll
             for (int n = 0; n < 16; ++n) {
               const int col = 8 * n + 2 * quad;

@@ -19,10 +19,13 @@ constexpr int kMaxNbs = 64;
 constexpr int kTileTok = 128;     // keys per attention tile (8 pages)
 constexpr int kAccMaxChunks = 16; // vocab chunks per row in the argmax
 constexpr int kTcRows = 64;       // rows of the tensor-core query tile (GQA group 4 x 16 slots)
-// Cost of one key tile in the attention schedule, by the request's window length: with more
-// than 8 live rows per q-head the second group of softmax warps works too and a tile takes
-// about 4.5 % longer (measured).  Slices are cut to equal cost, not to equal tile counts.
-constexpr int kTileCostSmall = 64, kTileCostBig = 67;
+// Cost model of the attention schedule (slices are cut to equal cost, not to equal tile counts),
+// fitted to per-CTA timestamps on the Qwen3-8B-shaped step: a key tile of a request with more than
+// 8 window rows takes about 6 % longer (the second group of softmax warps works too), a new
+// (request, kv-head) pair costs about 0.8 tile, and the last CTAs of a launch start 2-3 tiles late.
+constexpr int kTileCostSmall = 64, kTileCostBig = 68, kRunCost = 50;
+constexpr int kLateCtas = 8;
+__device__ constexpr int kLateTiles[kLateCtas] = {2, 2, 2, 2, 2, 2, 2, 3};
 // acceptance-predictor front end ("Acceptance predictor" paragraph)
 constexpr int kPredPos = 15;          // new draft positions per request
 constexpr int kPredConf = 18;         // confidence values per position
