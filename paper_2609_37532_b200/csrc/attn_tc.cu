@@ -66,6 +66,10 @@
 
 namespace dscale {
 
+#ifdef DSCALE_WAIT_TEST
+__device__ int g_drop_cta = -1, g_drop_tile = -1;
+#endif
+
 namespace {
 
 #ifndef DSCALE_PRODUCERS
@@ -89,7 +93,7 @@ constexpr int kOffQ = 0;                                 // 2 x 16 KB
 constexpr int kOffP = kOffQ + 2 * kQBytes;               // 2 x 16 KB
 constexpr int kOffKV = kOffP + 2 * kPBytes;              // 5 x 32 KB
 constexpr int kOffBar = kOffKV + kStages * kSlotBytes;   // mbarriers
-constexpr int kNumBars = 2 * kStages + 2 + 2 + 3 + 2 + 2 + 5;
+constexpr int kNumBars = 2 * kStages + 2 + 2 + 3 + 2 + 2 + 6;
 constexpr int kOffMisc = kOffBar + 8 * 32;               // tmem base, abort flag, tickets
 constexpr int kOffTile = kOffMisc + 64;                  // tile prefix, kMaxNbs + 1 ints
 constexpr int kOffSlice = kOffTile + (kMaxNbs + 1) * 4 + 12;   // slice starts, up to kMaxCtas + 1 ints
@@ -105,7 +109,8 @@ enum Bar { B_KV_FULL = 0, B_KV_EMPTY = kStages, B_Q_FULL = 2 * kStages, B_Q_EMPT
            B_PART = B_GROUP + 1,     // softmax -> publisher: the first run's partial is stored
            B_PUB = B_PART + 1,       // publisher -> softmax: that partial is published
            B_PARTNER = B_PUB + 1,    // producer -> softmax: partner partials landed (or not)
-           B_MERGE = B_PARTNER + 1 };// bulk copies of the end-phase merge
+           B_MERGE = B_PARTNER + 1,  // bulk copies of the end-phase merge
+           B_DRAIN = B_MERGE + 1 };  // products still in flight when a wait ran out
 
 // instruction descriptor: bf16 x bf16 -> fp32, M = 64, N = 128; B is K-major
 // for S = Q K^T and MN-major (tokens are the K dimension) for O = P V
@@ -169,6 +174,7 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
     mbar_init(bar(B_PUB), 1);
     mbar_init(bar(B_PARTNER), 1);
     mbar_init(bar(B_MERGE), 1);
+    mbar_init(bar(B_DRAIN), 1);
     *s_abort = 0;
     *s_dummy = 0;
     for (int x = 0; x < 4; ++x) s_lock[x] = 0;
@@ -265,6 +271,11 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           const int mine = min(kPagesPerProducer, max(0, n_pages - pw * kPagesPerProducer));   // pages of this warp
           if (lane == 0) mbar_expect_tx(bar(B_KV_FULL + slot), mine * kPageBytes);
           __syncwarp();
+#ifdef DSCALE_WAIT_TEST
+          // wait-limit test build only: the copies of one K tile of one CTA are left out (the
+          // barrier stays armed), so that every wait behind it runs into its limit
+          if (which == 0 && c == g_drop_cta && (int)(u / 2) == g_drop_tile) continue;
+#endif
           if (which == 0) {
             if (lane < 2 * kPagesPerProducer && pg_l < n_pages)
               tma_load_5d_hint(base + kOffKV + slot * kSlotBytes + k_half * kHalfSlot + pg_l * kPageHalf,
@@ -453,6 +464,13 @@ attn_tc_kernel(AttnArgs a, WsLayout L, const __grid_constant__ CUtensorMap tm_q,
           if (*s_abort) ok = false;
           else if (clock64() - t_idle > kWaitCycles) { *s_abort = 1; ok = false; }
         }
+      }
+      if (!ok) {
+        // A wait ran out somewhere in this CTA.  Products issued so far may still be running:
+        // tensor memory must not be released under them, so wait (bounded) for their completion.
+        if (leader) umma_commit(bar(B_DRAIN));
+        __syncwarp();
+        mbar_wait(bar(B_DRAIN), 0, s_dummy);
       }
     }
     __syncwarp();
@@ -950,3 +968,13 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t stream) {
 }
 
 }  // namespace dscale
+
+#ifdef DSCALE_WAIT_TEST
+// Wait-limit test build only: leave out the K copies of key tile `tile` (counted inside the
+// slice) of CTA `cta` in every following launch; (-1, -1) switches it off.  HOST call.
+extern "C" int dscale_test_drop_copy(int cta, int tile) {
+  if (cudaMemcpyToSymbol(dscale::g_drop_cta, &cta, sizeof(int)) != cudaSuccess) return -3;
+  if (cudaMemcpyToSymbol(dscale::g_drop_tile, &tile, sizeof(int)) != cudaSuccess) return -3;
+  return 0;
+}
+#endif

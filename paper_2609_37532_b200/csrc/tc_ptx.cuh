@@ -9,7 +9,12 @@
 namespace dscale {
 namespace {
 
-constexpr long long kWaitCycles = 1LL << 31;            // ~1 s bound on every wait
+// Bound on every device-side wait (about 1 s).  The wait-limit test library is the same code
+// built with a bound of about 1 ms (see build.py and tests/test_gpu_wait_limit.py).
+#ifndef DSCALE_WAIT_CYCLES
+#define DSCALE_WAIT_CYCLES (1LL << 31)
+#endif
+constexpr long long kWaitCycles = DSCALE_WAIT_CYCLES;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));

@@ -1,0 +1,108 @@
+"""A bounded device-side wait that runs out, made to happen without any GPU fault.
+
+Every wait inside the attention kernel (mbarrier waits of the copy, MMA and softmax warps)
+has a time limit; when one runs out the CTA raises its abort flag, all of its warps leave
+their loops, the copy warps wait (bounded) for the copies still in flight, the MMA warp waits
+(bounded) for the products still in flight, tensor memory is released and the kernel returns
+with DSCALE_STATUS_TIMEOUT set in the workspace.  Nothing traps and nothing spins without limit.
+
+The path is exercised with the wait-limit test build of the library
+(libdscale_waittest.so: the same sources, every limit at about 1 ms, plus a hook that leaves
+out the copies of one key tile of one CTA while the tile's barrier stays armed), loaded here
+beside the product library.  After the timed-out call the workspace is re-initialised, as the
+header prescribes for a sticky status, and the same call must match the oracle again.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from dscale_inputs import CONFIGS, small_variant
+from gpu_case import ALLOC_FIELDS, SCALE, attn_close, dev, full_case, oracle_attn
+
+pytestmark = pytest.mark.gpu
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+LIB_PATH = os.path.join(ROOT, "paper_2609_37532_b200", "libdscale_waittest.so")
+
+
+@pytest.fixture(scope="module")
+def wlib():
+    import paper_2609_37532_b200  # noqa: F401  (builds both libraries if they are stale)
+    lib = C.CDLL(LIB_PATH)
+    lib.dscale_workspace_bytes.restype = C.c_size_t
+    lib.dscale_ws_field.restype = C.c_void_p
+    lib.dscale_ws_field.argtypes = [C.c_void_p, C.c_int, C.c_int]
+    return lib
+
+
+def _vp(t):
+    return C.c_void_p(t.data_ptr())
+
+
+def test_a_wait_that_runs_out_sets_the_status_and_the_kernel_returns(wlib):
+    # two long pairs on two kv-heads: every CTA of the grid has a slice of a few key tiles
+    cfg = small_variant(CONFIGS["tiny"], n=2, seed=41)
+    req, alloc, kc, vc, qu, qp = full_case(cfg, ctx_override=[20000, 9000])
+    n_bs, hq, hkv = req["n_bs"], cfg.n_q_heads, cfg.n_kv_heads
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    nbytes = wlib.dscale_workspace_bytes(n_bs, hq, hkv, 128, sms)
+    buf = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    ws = buf.data_ptr() + (-buf.data_ptr()) % 256
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    n_live = dev(np.array([req["n_live"]], dtype=np.int32))
+    scores, draft = dev(req["scores"]), dev(req["draft_tokens"])
+    ctx, bt = dev(req["ctx_len"]), dev(req["block_table"])
+    q_d, k_d, v_d = qp.cuda(), kc.cuda(), vc.cuda()
+    out = torch.full(qp.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+
+    def status():
+        addr = wlib.dscale_ws_field(C.c_void_p(ws), n_bs, 0)
+        off = addr - buf.data_ptr()
+        return int(buf[off:off + 4].view(torch.int32).item())
+
+    def init_and_alloc():
+        assert wlib.dscale_workspace_init(C.c_void_p(ws), C.c_size_t(nbytes), n_bs, hq, hkv, 128, sms, stream) == 0
+        assert wlib.dscale_alloc_verify(C.c_void_p(ws), n_bs, _vp(n_live), _vp(scores), 0, _vp(draft), _vp(ctx),
+                                        _vp(bt), req["max_pages"], req["num_pages"], stream) == 0
+
+    def attention():
+        rc = wlib.dscale_verify_attn(C.c_void_p(ws), n_bs, _vp(q_d), _vp(k_d), _vp(v_d), _vp(bt), req["max_pages"],
+                                     req["num_pages"], hq, hkv, C.c_float(SCALE), _vp(out), stream)
+        assert rc == 0
+        torch.cuda.synchronize()          # returns: the kernel ended by itself
+
+    init_and_alloc()
+    torch.cuda.synchronize()
+    for f, fid in (("k", 1), ("offset", 2)):
+        addr = wlib.dscale_ws_field(C.c_void_p(ws), n_bs, fid)
+        off = addr - buf.data_ptr()
+        got = buf[off:off + 4 * len(alloc[f])].view(torch.int32).cpu().numpy()
+        np.testing.assert_array_equal(got, alloc[f], err_msg=f)
+
+    # 1. CTA 5 never gets the K copies of its second key tile: the waits behind it run out
+    assert wlib.dscale_test_drop_copy(5, 1) == 0
+    attention()
+    assert status() & 8, "DSCALE_STATUS_TIMEOUT was not set"
+    assert status() & ~8 == 0
+
+    # 2. the status is sticky, and the pair whose contributor gave up never completed its
+    #    ticket count: the workspace is initialised again, as the header prescribes
+    assert wlib.dscale_test_drop_copy(-1, -1) == 0
+    init_and_alloc()
+    out.fill_(float("nan"))
+    attention()
+    assert status() == 0
+    ok, max_abs, worst = attn_close(out, oracle_attn(req, alloc, kc, vc, qp))
+    assert ok, f"after re-initialisation: max|d|={max_abs} at {worst}"
+
+    # 3. and once more without re-initialising: the tickets of a clean launch reset themselves
+    out.fill_(float("nan"))
+    attention()
+    assert status() == 0
+    ok, max_abs, worst = attn_close(out, oracle_attn(req, alloc, kc, vc, qp))
+    assert ok, f"second clean launch: max|d|={max_abs} at {worst}"
+    assert wlib.dscale_workspace_destroy(C.c_void_p(ws)) == 0
