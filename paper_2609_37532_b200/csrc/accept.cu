@@ -1,18 +1,21 @@
 // Greedy prefix verification: vocabulary argmax per packed row, then the
 // accepted-prefix scan per request, in one launch.
 //
-// The argmax is a pure HBM stream (8N rows x vocab fp32 read once).  The grid
-// is (vocab chunks, 8 n_bs rows); a block streams its chunk with 128-bit
-// read-only loads that bypass L1, up to eight loads in flight per thread, keeps a
-// per-thread running (max, first index), reduces it with warp shuffles and
-// writes one partial to the workspace.  The last block to finish (a ticket in
-// the workspace header, no waiting) merges the partials in chunk order and
+// The argmax is a pure HBM stream (8N rows x vocab fp32 read once).  The live logits are
+// taken as one ragged sequence of 16-byte vectors (row-major, ceil(vocab / 4) per row) and cut
+// into one equal span per warp of a grid of two 512-thread CTAs per SM: every warp streams
+// its span with 128-bit read-only loads that bypass L1, eight in flight per lane (128 KB in
+// flight per SM), keeps a per-thread running (max, first index), and at the end of a row
+// segment reduces it with warp shuffles and folds it into the row's 64-bit key in the
+// workspace with one atomicMax: key = (order-preserving bits of the value, ~index), so that the
+// largest key is the largest value and, among equal values, the lowest index.  A NaN or
+// -inf is never offered, an untouched key (0) means token 0.  No partial arrays, no block
+// barrier in the stream.  The last CTA to finish (a ticket in the workspace header, no
+// waiting) turns the keys into target tokens, clears them for the next launch, and
 // runs the sequential acceptance loop of the "Prefix verifier" paragraph with
 // one thread per request (on shared-memory copies of the row results and the
-// packed tokens), writing the outputs of Algorithm 2, lines 21-26.  (One warp
-// per (row, chunk) without any block barrier was tried and is slower: 49 vs 39 us.)
-// Rows at or beyond M_live = 8N (read on the device) exit immediately, so the
-// same captured launch serves every N <= n_bs.
+// packed tokens), writing the outputs of Algorithm 2, lines 21-26.
+// M_live is read on the device, so the same captured launch serves every N <= n_bs.
 #include <cfloat>
 #include <climits>
 
@@ -22,7 +25,7 @@ namespace dscale {
 
 namespace {
 
-constexpr int kAccThreads = 256;
+constexpr int kAccThreads = 512;
 
 struct Best {
   float v;
@@ -47,79 +50,69 @@ __device__ __forceinline__ float4 ldg_stream(const float4* p) {
   return r;
 }
 
-__global__ void __launch_bounds__(kAccThreads) accept_kernel(AcceptArgs a, WsLayout L, int chunks,
-                                                             int chunk_len) {
+__device__ __forceinline__ unsigned long long key_of(float v, int i) {
+  unsigned u = v == 0.0f ? 0u : __float_as_uint(v);    // -0 and +0 are one value
+  u ^= (u >> 31) ? 0xffffffffu : 0x80000000u;          // unsigned order = float order
+  return ((unsigned long long)u << 32) | (unsigned)(~i);
+}
+
+__global__ void __launch_bounds__(kAccThreads, 2) accept_kernel(AcceptArgs a, WsLayout L) {
   int* hdr = ws_ptr<int>(a.ws, L.hdr);
   const int m_live = hdr[H_M_LIVE];
-  const int s = blockIdx.y;
-  if (s >= m_live) return;
-  const int c = blockIdx.x;
-  const int tid = threadIdx.x;
-  float* pval = ws_ptr<float>(a.ws, L.amax_val);
-  int* pidx = ws_ptr<int>(a.ws, L.amax_idx);
+  const int tid = threadIdx.x, lane = tid & 31;
+  unsigned long long* row_key = ws_ptr<unsigned long long>(a.ws, L.amax_val);   // [8 n_bs], 0 = untouched
+  __shared__ int sLast;
 
-  const float* row = a.logits + (size_t)s * a.ld;
-  const int lo = c * chunk_len;
-  const int hi = min(a.vocab, lo + chunk_len);
-  Best b{-INFINITY, INT_MAX};
-  if (lo < hi) {
-    const int n4 = (hi - lo) >> 2;                  // chunk_len % 4 == 0, row 16-byte aligned
-    const float4* p4 = reinterpret_cast<const float4*>(row + lo);
-    int x = tid;
-    for (; x + 7 * kAccThreads < n4; x += 8 * kAccThreads) {      // eight 128-bit loads in flight
+  // this warp's span of the ragged vector sequence
+  const long long nv = (a.vocab + 3) >> 2;                      // vectors per row
+  const long long total = nv * m_live;
+  const long long n_warps = (long long)gridDim.x * (kAccThreads / 32);
+  const long long w = (long long)blockIdx.x * (kAccThreads / 32) + (tid >> 5);
+  long long pos = total * w / n_warps;
+  const long long end = total * (w + 1) / n_warps;
+  while (pos < end) {
+    const int s = (int)(pos / nv);
+    const int v0 = (int)(pos - (long long)s * nv);
+    const int v1 = (int)min(nv, v0 + (end - pos));                // segment [v0, v1) of row s
+    const float4* p4 = reinterpret_cast<const float4*>(a.logits + (size_t)s * a.ld);
+    const bool ragged = (a.vocab & 3) && v1 == nv;                // the row's last vector is partly padding
+    const int v1_full = ragged ? v1 - 1 : v1;
+    Best b{-INFINITY, INT_MAX};
+    int x = v0 + lane;
+    for (; x + 7 * 32 < v1_full; x += 8 * 32) {                   // eight 128-bit loads in flight
       float4 v[8];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) v[q] = ldg_stream(p4 + x + q * kAccThreads);
+      for (int q = 0; q < 8; ++q) v[q] = ldg_stream(p4 + x + q * 32);
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
-        const int e = lo + 4 * (x + q * kAccThreads);
+        const int e = 4 * (x + q * 32);
         take(b, v[q].x, e); take(b, v[q].y, e + 1); take(b, v[q].z, e + 2); take(b, v[q].w, e + 3);
       }
     }
-    for (; x + 3 * kAccThreads < n4; x += 4 * kAccThreads) {
-      float4 v0 = ldg_stream(p4 + x);
-      float4 v1 = ldg_stream(p4 + x + kAccThreads);
-      float4 v2 = ldg_stream(p4 + x + 2 * kAccThreads);
-      float4 v3 = ldg_stream(p4 + x + 3 * kAccThreads);
-      int e = lo + 4 * x;
-      take(b, v0.x, e); take(b, v0.y, e + 1); take(b, v0.z, e + 2); take(b, v0.w, e + 3);
-      e += 4 * kAccThreads;
-      take(b, v1.x, e); take(b, v1.y, e + 1); take(b, v1.z, e + 2); take(b, v1.w, e + 3);
-      e += 4 * kAccThreads;
-      take(b, v2.x, e); take(b, v2.y, e + 1); take(b, v2.z, e + 2); take(b, v2.w, e + 3);
-      e += 4 * kAccThreads;
-      take(b, v3.x, e); take(b, v3.y, e + 1); take(b, v3.z, e + 2); take(b, v3.w, e + 3);
+    for (; x < v1_full; x += 32) {
+      const float4 v = ldg_stream(p4 + x);
+      const int e = 4 * x;
+      take(b, v.x, e); take(b, v.y, e + 1); take(b, v.z, e + 2); take(b, v.w, e + 3);
     }
-    for (; x < n4; x += kAccThreads) {
-      float4 v0 = ldg_stream(p4 + x);
-      const int e = lo + 4 * x;
-      take(b, v0.x, e); take(b, v0.y, e + 1); take(b, v0.z, e + 2); take(b, v0.w, e + 3);
+    if (ragged && lane == 0) {
+      const float* row = a.logits + (size_t)s * a.ld;
+      for (int e = 4 * v1_full; e < a.vocab; ++e) take(b, row[e], e);
     }
-    for (int e = lo + 4 * n4 + tid; e < hi; e += kAccThreads) take(b, row[e], e);
-  }
-  // warp-shuffle reduction, then across the 8 warps
 #pragma unroll
-  for (int d = 16; d > 0; d >>= 1) {
-    Best o{__shfl_xor_sync(0xffffffffu, b.v, d), __shfl_xor_sync(0xffffffffu, b.i, d)};
-    b = merge(b, o);
+    for (int d = 16; d > 0; d >>= 1) {
+      Best o{__shfl_xor_sync(0xffffffffu, b.v, d), __shfl_xor_sync(0xffffffffu, b.i, d)};
+      b = merge(b, o);
+    }
+    if (lane == 0 && b.i != INT_MAX) atomicMax(&row_key[s], key_of(b.v, b.i));
+    pos += v1 - v0;
   }
-  __shared__ float sv[kAccThreads / 32];
-  __shared__ int si[kAccThreads / 32];
-  __shared__ int sLast;
-  if ((tid & 31) == 0) { sv[tid >> 5] = b.v; si[tid >> 5] = b.i; }
+  __threadfence();
   __syncthreads();
-  if (tid == 0) {
-    for (int w = 1; w < kAccThreads / 32; ++w) b = merge(b, Best{sv[w], si[w]});
-    pval[(size_t)s * kAccMaxChunks + c] = b.v;
-    pidx[(size_t)s * kAccMaxChunks + c] = b.i;
-    __threadfence();
-    const int ticket = atomicAdd(&hdr[H_ACCEPT_TICKET], 1);
-    sLast = (ticket == chunks * m_live - 1);
-  }
+  if (tid == 0) sLast = (atomicAdd(&hdr[H_ACCEPT_TICKET], 1) == (int)gridDim.x - 1);
   __syncthreads();
   if (!sLast) return;
 
-  // ---- last block: merge partials, then the acceptance loop ----------------
+  // ---- last block: keys -> target tokens, then the acceptance loop ----------
   __threadfence();
   if (tid == 0) hdr[H_ACCEPT_TICKET] = 0;           // ready for the next replay
   const int n_bs = a.n_bs;
@@ -133,13 +126,9 @@ __global__ void __launch_bounds__(kAccThreads) accept_kernel(AcceptArgs a, WsLay
   for (int r = tid; r < m_bs; r += kAccThreads) {
     int best = 0;
     if (r < m_live) {
-      Best bb{-INFINITY, INT_MAX};
-      for (int cc = 0; cc < chunks; ++cc) {
-        Best o{__ldcg(&pval[(size_t)r * kAccMaxChunks + cc]),
-               __ldcg(&pidx[(size_t)r * kAccMaxChunks + cc])};
-        bb = merge(bb, o);
-      }
-      best = bb.i == INT_MAX ? 0 : bb.i;            // row without any finite / -inf-beating entry
+      const unsigned long long key = __ldcg(&row_key[r]);
+      if (key != 0ull) best = (int)~(unsigned)(key & 0xffffffffull);   // untouched: no entry beat -inf
+      row_key[r] = 0ull;                            // ready for the next replay
     }
     top1[r] = best;
     s_top1[r] = best;
@@ -175,12 +164,11 @@ __global__ void __launch_bounds__(kAccThreads) accept_kernel(AcceptArgs a, WsLay
 
 cudaError_t launch_accept(const AcceptArgs& a, cudaStream_t stream) {
   WsLayout L = ws_layout(a.n_bs, a.n_kv_heads, a.num_ctas);
-  int chunks = a.vocab / 16384;
-  chunks = chunks < 1 ? 1 : (chunks > kAccMaxChunks ? kAccMaxChunks : chunks);
-  int chunk_len = (a.vocab + chunks - 1) / chunks;
-  chunk_len = (chunk_len + 3) & ~3;
-  dim3 grid(chunks, kHalfW * a.n_bs);
-  accept_kernel<<<grid, kAccThreads, 0, stream>>>(a, L, chunks, chunk_len);
+  // two CTAs per SM; small problems get fewer, so that a warp's span is at least 4 KB
+  const long long vecs = (long long)((a.vocab + 3) >> 2) * kHalfW * a.n_bs;
+  long long ctas = vecs / (256 * (kAccThreads / 32));
+  ctas = ctas < 1 ? 1 : (ctas > 2LL * a.num_ctas ? 2LL * a.num_ctas : ctas);
+  accept_kernel<<<dim3((unsigned)ctas), kAccThreads, 0, stream>>>(a, L);
   return cudaGetLastError();
 }
 
