@@ -135,6 +135,21 @@ __device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// offer the four values of every lane: the lane maxima first (one round), and the other three
+// only if one of them still beats the 16th afterwards (an event usually brings a single value)
+__device__ __forceinline__ void top16_offer_vec(float& tv, float& tau, float4 z, float zmax, int lane) {
+  if (!__any_sync(0xffffffffu, zmax > tau)) return;
+  top16_offer(tv, tau, zmax, lane);
+  // the remaining three: the first component equal to the maximum is the one already offered
+  const bool mx = z.x == zmax, my = !mx && z.y == zmax, mz = !mx && !my && z.z == zmax;
+  const float rx = mx ? -INFINITY : z.x, ry = my ? -INFINITY : z.y, rz = mz ? -INFINITY : z.z;
+  const float rw = (mx || my || mz) ? z.w : -INFINITY;
+  if (__any_sync(0xffffffffu, fmaxf(fmaxf(rx, ry), fmaxf(rz, rw)) > tau)) {
+    top16_offer(tv, tau, rx, lane); top16_offer(tv, tau, ry, lane);
+    top16_offer(tv, tau, rz, lane); top16_offer(tv, tau, rw, lane);
+  }
+}
+
 // running statistics of one logit row in one lane
 struct RowStat {
   float m2, s, t, zsum;      // m2 = running max times log2(e)
@@ -204,10 +219,8 @@ __device__ __forceinline__ void row_update2(RowStat& a, RowStat& b, float4 za, f
     a.zsum += xa[x]; b.zsum += xb[x];
   }
   if (__any_sync(0xffffffffu, la > a.tau || lb > b.tau)) {  // rare once the lists have warmed up
-    top16_offer(a.tv, a.tau, za.x, lane); top16_offer(a.tv, a.tau, za.y, lane);
-    top16_offer(a.tv, a.tau, za.z, lane); top16_offer(a.tv, a.tau, za.w, lane);
-    top16_offer(b.tv, b.tau, zb.x, lane); top16_offer(b.tv, b.tau, zb.y, lane);
-    top16_offer(b.tv, b.tau, zb.z, lane); top16_offer(b.tv, b.tau, zb.w, lane);
+    top16_offer_vec(a.tv, a.tau, za, la, lane);
+    top16_offer_vec(b.tv, b.tau, zb, lb, lane);
   }
 }
 
