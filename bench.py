@@ -136,6 +136,30 @@ def algorithmic_bytes(cfg, req, k):
     return per_layer, logits + small
 
 
+def step_bytes_of(cfg, req):
+    """Algorithmic bytes of one step; needs no allocation (the lengths sum to 8 N)."""
+    n = req["n_live"]
+    kv_tok = int(req["ctx_len"][:n].astype(np.int64).sum()) + 8 * n
+    pages = int(((req["ctx_len"][:n].astype(np.int64) + 8 + 15) // 16).sum())     # about: lengths vary around 8
+    per_layer = kv_tok * cfg.n_kv_heads * 128 * 2 * 2 + pages * 4 + 2 * 8 * n * cfg.n_q_heads * 128 * 2
+    return per_layer * cfg.layers + 8 * n * cfg.vocab * 4
+
+
+def workload_config(cfg, req, attn="tensor"):
+    """The `config` object of the JSON line: the same for both arms (the reference arm times the
+    CPU oracle on a sample of exactly this workload)."""
+    n = req["n_live"]
+    sb = step_bytes_of(cfg, req)
+    flush = sb < 4 * L2_BYTES
+    return {"workload": cfg.name, "requests_per_gpu": n, "layers": cfg.layers,
+            "heads": [cfg.n_q_heads, cfg.n_kv_heads], "ctx": [cfg.ctx_lo, cfg.ctx_hi],
+            "vocab": cfg.vocab, "packed_rows": 8 * n, "attn": attn,
+            "l2": ("inputs_larger_than_L2 (%.1f GB per step)" % (sb / 1e9)) if not flush else
+                  ("L2 flushed before every timed replay (a %d MB buffer rewritten; %.1f MB per step); "
+                   "step time = sum of the per-replay intervals" % (FLUSH_BYTES >> 20, sb / 1e6)),
+            "launch": "one captured CUDA graph per step"}
+
+
 # ------------------------------------------------------------------ CPU oracle
 def oracle_step_sample(cfg, req, kvs, q_unpacked, logits_unpacked):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload:
@@ -203,8 +227,7 @@ def run_reference(args, rank):
         "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * work / max(1, args.steps), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": cfg.name, "requests": cfg.n, "layers": cfg.layers,
-                   "ctx": [cfg.ctx_lo, cfg.ctx_hi], "vocab": cfg.vocab},
+        "config": workload_config(cfg, req),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -544,13 +567,7 @@ def run_ours(args, rank, world, local_rank):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "requests_per_gpu": n, "layers": cfg.layers,
-                       "heads": [cfg.n_q_heads, cfg.n_kv_heads], "ctx": [cfg.ctx_lo, cfg.ctx_hi],
-                       "vocab": cfg.vocab, "packed_rows": 8 * n, "attn": args.attn,
-                       "l2": ("inputs_larger_than_L2 (%.1f GB per step)" % (step_bytes / 1e9)) if not flush else
-                             ("L2 flushed before every timed replay (a %d MB buffer rewritten; %.1f MB per step); "
-                              "step time = sum of the per-replay intervals" % (FLUSH_BYTES >> 20, step_bytes / 1e6)),
-                       "launch": "one captured CUDA graph per step"},
+            "config": workload_config(cfg, req, args.attn),
             "verified_tokens_per_step": tokens_per_step,
             "step_ms": {"mean": ms_step, "median": float(np.median(per_replay)), "min": float(per_replay.min()),
                         "warm_median": warm_ms},
