@@ -346,6 +346,20 @@ def run_ours(args, rank, world, local_rank):
         barrier()
         return np.array([evs[2 * s_].elapsed_time(evs[2 * s_ + 1]) for s_ in range(count)])
 
+    def time_captured(fn, inner=8, reps=None):
+        """Per-call device time in ms of fn(): `inner` calls captured as one graph (what a step
+        does with every call of this library), median over the replays."""
+        fn()
+        barrier()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(inner):
+                fn()
+        g.replay()
+        barrier()
+        reps = reps or max(5, min(args.steps, 20))
+        return float(np.median(timed_replays(g, reps, cold=False))) / inner
+
     sampler = ClockSampler(local_rank)
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
@@ -385,23 +399,13 @@ def run_ours(args, rank, world, local_rank):
         attn_ms = float(np.mean(_per))
         attn_med_ms, attn_min_ms = float(np.median(_per)), float(_per.min())
         ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ea.record(stream)
-        for _ in range(args.steps):
-            do_accept()
-        eb.record(stream)
-        barrier()
-        accept_ms = ea.elapsed_time(eb) / args.steps
+        accept_ms = time_captured(do_accept)
         # the sampling verifier (temperature 1) on the same logits, for its own figure
         u_acc = torch.rand(8 * n_bs, device=dev)
         u_drw = torch.rand(n_bs, device=dev)
         so = [torch.zeros_like(outs[0]), torch.zeros_like(outs[1]), torch.zeros_like(outs[2]), torch.zeros_like(outs[3])]
-        P.accept_sampling(ws, logits, cfg.vocab, 1.0, u_acc, u_drw, so[0], so[1], so[2], so[3])
-        ea.record(stream)
-        for _ in range(args.steps):
-            P.accept_sampling(ws, logits, cfg.vocab, 1.0, u_acc, u_drw, so[0], so[1], so[2], so[3])
-        eb.record(stream)
-        barrier()
-        sampling_ms = ea.elapsed_time(eb) / args.steps
+        sampling_ms = time_captured(
+            lambda: P.accept_sampling(ws, logits, cfg.vocab, 1.0, u_acc, u_drw, so[0], so[1], so[2], so[3]))
 
         # the fused LM head + argmax + acceptance (one launch) on seeded hidden states
         lm = None
@@ -410,14 +414,7 @@ def run_ours(args, rank, world, local_rank):
             h_lm = rows_to_packed(h_un, k, offset, n, 8 * n_bs)
             del h_un
             lo = [torch.zeros_like(x) for x in outs[:4]]
-            for _ in range(3):
-                P.lm_head_accept(ws, h_lm, w_lm, lo[0], lo[1], lo[2], lo[3])
-            ea.record(stream)
-            for _ in range(args.steps):
-                P.lm_head_accept(ws, h_lm, w_lm, lo[0], lo[1], lo[2], lo[3])
-            eb.record(stream)
-            barrier()
-            lm_ms = ea.elapsed_time(eb) / args.steps
+            lm_ms = time_captured(lambda: P.lm_head_accept(ws, h_lm, w_lm, lo[0], lo[1], lo[2], lo[3]), inner=4)
             # context: the library GEMM that would only produce the logits (bf16 out)
             for _ in range(2):
                 lg = torch.matmul(h_lm, w_lm.t())
@@ -446,14 +443,7 @@ def run_ours(args, rank, world, local_rank):
             def do_pred():
                 P.predict_scores(ws, d_n_live, pin["draft_logits"], cfg.vocab, pin["draft_hidden"], pin["p_hidden"],
                                  pin["p_logit"], pin["w1"], pin["b1"], pin["w2"], pin["b2"], pl_out)
-            for _ in range(3):
-                do_pred()
-            ea.record(stream)
-            for _ in range(args.steps):
-                do_pred()
-            eb.record(stream)
-            barrier()
-            pred_ms = ea.elapsed_time(eb) / args.steps
+            pred_ms = time_captured(do_pred, inner=4)
             pred_bytes = 15 * n * cfg.vocab * 4 + 32 * cfg.vocab * 2 + 15 * n * args.pred_hidden * 2
             pred = {"us": pred_ms * 1e3, "hidden": args.pred_hidden, "bytes": pred_bytes,
                     "gbs": pred_bytes / (pred_ms * 1e-3) / 1e9,
