@@ -7,7 +7,7 @@ steps at the same addresses:
 Each stage is compared with the oracle on the inputs it actually saw: the predictor's
 predLogits within their tolerance; the allocation bit-exactly against the oracle run on the
 device's own predLogits (an integer decision is only ever compared on identical scores);
-attention within 1e-2 + 1e-2|ref|; the LM-head tokens by the margin rule of
+attention within the bounds of gpu_case.attn_close; the LM-head tokens by the margin rule of
 test_gpu_lm_head.py and the acceptance outputs against the sequential loop on those tokens."""
 import numpy as np
 import pytest

@@ -1,6 +1,8 @@
 """GPU parity: the CUDA library (through its C ABI) against the CPU oracle,
 element by element, on the same seeded inputs.  Integer results must be
-bit-exact; bf16 attention outputs must satisfy |gpu - ref| <= 1e-2 + 1e-2 |ref|.
+bit-exact; bf16 attention outputs must satisfy |gpu - ref| <= max(1e-2, 1e-2 |ref|)
+per element and, per (row, q-head) vector, |gpu - ref|_2 <= 8e-3 |ref|_2 + 2e-4
+(gpu_case.attn_close).
 """
 import numpy as np
 import pytest
