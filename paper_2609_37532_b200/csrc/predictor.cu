@@ -1,7 +1,7 @@
 // Acceptance-predictor front end: drafter logits and hidden states -> 1735
 // features -> 1735-64-15 perceptron -> predLogits ("Acceptance predictor"
-// paragraph, Eq. 4 and Eq. 5).  Four launches (the hidden-state projection goes first and
-// overlaps with the logit stream):
+// paragraph, Eq. 4 and Eq. 5).  Three launches (the hidden-state projection goes first and
+// overlaps with the logit stream; the tail is scheduled while the stream runs):
 //
 //  pred_stream_kernel    the only pass over the drafter logits (15 N rows x V fp32,
 //                        292 MB at N = 32: an HBM stream).  A CTA of 16 warps owns
@@ -20,11 +20,11 @@
 //                        along with a 292 MB stream, there is no tensor-core
 //                        time to win, and the rows are already in registers.
 //                        One record per (row, chunk) goes to the workspace.
-//  pred_features_kernel  per request: merges the chunk records into the 18
-//                        confidence values and the centred logit projection per
-//                        position, appends the batch context.
 //  pred_hidden_kernel    the 64 x H hidden-state projection of all rows (bf16 MMAs).
-//  pred_mlp_kernel       per request: relu(W1 f + b1), W2 h + b2.
+//  pred_tail_kernel      per request: merges the chunk records into the 18
+//                        confidence values and the centred logit projection per
+//                        position, appends the hidden projection and the batch
+//                        context, then relu(W1 f + b1), W2 h + b2.
 #include <cfloat>
 #include <climits>
 #include <cuda_bf16.h>
@@ -241,6 +241,9 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
   auto empty = [&](int st) { return sbase + kOffBar + 8u * (kStages + st); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // the tail kernel behind this one may be scheduled now: it touches nothing this grid writes
+  // before its own wait on this grid's completion
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   int n = *a.n_live;
   n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
   const int live_rows = kPredPos * n;
@@ -470,73 +473,6 @@ struct FeatArgs {
   float* feat;                     // [n_bs][1735]
 };
 
-constexpr int kFeatThreads = 512;   // one warp per draft position
-
-__global__ void __launch_bounds__(kFeatThreads) pred_features_kernel(FeatArgs a) {
-  const int i = blockIdx.x;
-  int n = *a.n_live;
-  n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
-  if (i >= n) return;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  float* f = a.feat + (size_t)i * kPredFeatures;
-
-  {
-    // ---- confidence values and centred logit projection, one warp per position
-    for (int p = warp; p < kPredPos; p += kFeatThreads / 32) {
-      const int row = i * kPredPos + p;
-      const float* rec0 = a.part + (size_t)row * a.chunks * kPredRec;
-      // all loads of this position first (independent), then the merges
-      float cand[kPredMaxChunks / 2];                       // lane l: candidate l % 16 of chunk 2 x + l / 16
-#pragma unroll
-      for (int x = 0; x < kPredMaxChunks / 2; ++x) {
-        const int c = 2 * x + (lane >> 4);
-        cand[x] = c < a.chunks ? rec0[(size_t)c * kPredRec + (lane & 15)] : -INFINITY;
-      }
-      float proj = 0.f, rs = 0.f;
-#pragma unroll 8
-      for (int c = 0; c < a.chunks; ++c) {
-        proj += rec0[(size_t)c * kPredRec + 20 + lane];
-        rs += a.rowsum[c * kPredLog + lane];
-      }
-      const float pivot = a.logits[(size_t)row * a.ld];
-      float tv = -INFINITY, tau = -INFINITY;
-#pragma unroll
-      for (int x = 0; x < kPredMaxChunks / 2; ++x)
-        if (2 * x < a.chunks) top16_offer(tv, tau, cand[x], lane);
-      // merge the chunks' (max, sum, sum e z, sum z): lane = chunk
-      float m = -INFINITY, s_sum = 0.f, t_sum = 0.f, z_sum = 0.f;
-      if (lane < a.chunks) {
-        const float* r = rec0 + (size_t)lane * kPredRec;
-        m = r[16]; s_sum = r[17]; t_sum = r[18]; z_sum = r[19];
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
-        const float s2 = __shfl_xor_sync(0xffffffffu, s_sum, o);
-        const float t2 = __shfl_xor_sync(0xffffffffu, t_sum, o);
-        z_sum += __shfl_xor_sync(0xffffffffu, z_sum, o);
-        const float mm = fmaxf(m, m2);
-        const float r1 = m == -INFINITY ? 0.f : expf(m - mm), r2 = m2 == -INFINITY ? 0.f : expf(m2 - mm);
-        s_sum = s_sum * r1 + s2 * r2;
-        t_sum = t_sum * r1 + t2 * r2;
-        m = mm;
-      }
-      const float lse = m + logf(s_sum);
-      const float top = __shfl_sync(0xffffffffu, tv, 0);
-      float* fc = f + p * kPredConf;
-      if (lane == 0) fc[0] = top;
-      else if (lane < 16) fc[lane] = top - tv;
-      else if (lane == 16) fc[16] = top - lse;
-      else if (lane == 17) fc[17] = lse - t_sum / s_sum;
-      // logit projection of z - mean(z): the kernel accumulated P (z - pivot)
-      const float mean = z_sum / (float)a.vocab;
-      f[kPredPos * (kPredConf + kPredHid) + p * kPredLog + lane] = proj - (mean - pivot) * rs;
-    }
-    if (warp == 0 && lane < kPredCtx)
-      f[kPredFeatures - kPredCtx + lane] = lane == 0 ? (float)n : (lane == 3 ? 1.f : 0.f);
-  }
-}
-
 // ---------------------------------------------------------------------------
 // Hidden-state projection: [15 N rows x H] . [H x 64], a small dense contraction
 // (0.25 GFLOP at N = 32, H = 4096) on warp-level bf16 MMAs.  A CTA owns 16 rows;
@@ -624,33 +560,128 @@ struct MlpArgs {
   float* features_out;  // nullable [n_bs][1735]
 };
 
-constexpr int kMlpThreads = 1024;                           // 32 warps: two hidden units each
+// ---------------------------------------------------------------------------
+// Per request, behind the stream: merge the chunk records into the 18 confidence values and the
+// centred logit projection of each position, append the hidden-state projection and the batch
+// context, then relu(W1 f + b1) and W2 h + b2.  One launch (the merge and the perceptron used to
+// be two, each paying a launch and a cold pass over its inputs); it is launched with
+// programmatic stream serialisation: everything that depends only on the call's inputs (the
+// pivots, pulling W1 into L2 with an evict-last hint while the logit stream is still running)
+// happens before the grid dependency is waited for.
+constexpr int kTailThreads = 1024;                          // 32 warps: a position each, then two hidden units each
 
-__global__ void __launch_bounds__(kMlpThreads) pred_mlp_kernel(MlpArgs a) {
+// order-preserving key of a float for integer warp reductions; a NaN gets the lowest key
+__device__ __forceinline__ unsigned f2key(float v) {
+  const unsigned u = __float_as_uint(v);
+  return v == v ? (u ^ ((u >> 31) ? 0xffffffffu : 0x80000000u)) : 0u;
+}
+__device__ __forceinline__ float key2f(unsigned k) {
+  return __uint_as_float(k ^ ((k >> 31) ? 0x80000000u : 0xffffffffu));
+}
+
+__global__ void __launch_bounds__(kTailThreads, 1) pred_tail_kernel(FeatArgs a, MlpArgs m) {
   __shared__ float sf[kPredFeatures];
   __shared__ float sh[kPredMlp];
   const int i = blockIdx.x;
   int n = *a.n_live;
   n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (i >= n) {                                           // dead request: zeros
-    if (tid < kPredPos) a.pred_logits[i * kPredPos + tid] = 0.f;
-    if (a.features_out)
-      for (int x = tid; x < kPredFeatures; x += kMlpThreads) a.features_out[(size_t)i * kPredFeatures + x] = 0.f;
+  const bool live = i < n;
+  // ---- before the grid dependency: inputs of the call only
+  float pivot = 0.f;
+  if (live) {
+    for (int x = tid * 32; x < kPredMlp * kPredFeatures; x += kTailThreads * 32)
+      asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(m.w1 + x));
+    if (warp < kPredPos) pivot = a.logits[(size_t)(i * kPredPos + warp) * a.ld];
+  }
+  pdl_wait();
+  if (!live) {                                              // dead request: zeros
+    if (tid < kPredPos) m.pred_logits[i * kPredPos + tid] = 0.f;
+    if (m.features_out)
+      for (int x = tid; x < kPredFeatures; x += kTailThreads) m.features_out[(size_t)i * kPredFeatures + x] = 0.f;
     return;
   }
-  for (int x = tid; x < kPredFeatures; x += kMlpThreads) {
-    const float v = a.feat[(size_t)i * kPredFeatures + x];
-    sf[x] = v;
-    if (a.features_out) a.features_out[(size_t)i * kPredFeatures + x] = v;
+  if (warp < kPredPos) {
+    // ---- confidence values and centred logit projection, one warp per position
+    const int p = warp;
+    const int row = i * kPredPos + p;
+    const float* rec0 = a.part + (size_t)row * a.chunks * kPredRec;
+    // all loads of this position first (independent), then the merges
+    unsigned cand[kPredMaxChunks / 2];                      // lane l: candidate l % 16 of chunk 2 x + l / 16
+#pragma unroll
+    for (int x = 0; x < kPredMaxChunks / 2; ++x) {
+      const int c = 2 * x + (lane >> 4);
+      cand[x] = c < a.chunks ? f2key(rec0[(size_t)c * kPredRec + (lane & 15)]) : 0u;
+    }
+    float proj = 0.f, rs = 0.f;
+#pragma unroll 8
+    for (int c = 0; c < a.chunks; ++c) {
+      proj += rec0[(size_t)c * kPredRec + 20 + lane];
+      rs += a.rowsum[c * kPredLog + lane];
+    }
+    float mx = -INFINITY, s_sum = 0.f, t_sum = 0.f, z_sum = 0.f;   // the chunks' (max, sum, sum e z, sum z): lane = chunk
+    if (lane < a.chunks) {
+      const float* r = rec0 + (size_t)lane * kPredRec;
+      mx = r[16]; s_sum = r[17]; t_sum = r[18]; z_sum = r[19];
+    }
+    // the 16 largest of all chunks' candidates, in order: sixteen rounds of (lane maximum, warp
+    // maximum by an integer reduction, the first lane holding it gives it up)
+    float tv = -INFINITY;                                   // lane j < 16: the (j + 1)-th largest
+#pragma unroll 1
+    for (int j = 0; j < 16; ++j) {
+      unsigned lm = 0u;
+#pragma unroll
+      for (int x = 0; x < kPredMaxChunks / 2; ++x)
+        if (2 * x < a.chunks) lm = max(lm, cand[x]);
+      const unsigned gm = __reduce_max_sync(0xffffffffu, lm);
+      const unsigned who = __ballot_sync(0xffffffffu, lm == gm);
+      if (lane == __ffs(who) - 1) {
+        bool gone = false;
+#pragma unroll
+        for (int x = 0; x < kPredMaxChunks / 2; ++x)
+          if (2 * x < a.chunks && !gone && cand[x] == gm) { cand[x] = 0u; gone = true; }
+      }
+      if (lane == j) tv = gm != 0u ? key2f(gm) : -INFINITY;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, mx, o);
+      const float s2 = __shfl_xor_sync(0xffffffffu, s_sum, o);
+      const float t2 = __shfl_xor_sync(0xffffffffu, t_sum, o);
+      z_sum += __shfl_xor_sync(0xffffffffu, z_sum, o);
+      const float mm = fmaxf(mx, m2);
+      const float r1 = mx == -INFINITY ? 0.f : expf(mx - mm), r2 = m2 == -INFINITY ? 0.f : expf(m2 - mm);
+      s_sum = s_sum * r1 + s2 * r2;
+      t_sum = t_sum * r1 + t2 * r2;
+      mx = mm;
+    }
+    const float lse = mx + logf(s_sum);
+    const float top = __shfl_sync(0xffffffffu, tv, 0);
+    float* fc = sf + p * kPredConf;
+    if (lane == 0) fc[0] = top;
+    else if (lane < 16) fc[lane] = top - tv;
+    else if (lane == 16) fc[16] = top - lse;
+    else if (lane == 17) fc[17] = lse - t_sum / s_sum;
+    // logit projection of z - mean(z): the stream accumulated P (z - pivot)
+    const float mean = z_sum / (float)a.vocab;
+    sf[kPredPos * (kPredConf + kPredHid) + p * kPredLog + lane] = proj - (mean - pivot) * rs;
+  } else {
+    // ---- the other warps: the hidden-state projection of this request and the batch context
+    const float* hsrc = a.feat + (size_t)i * kPredFeatures + kPredPos * kPredConf;
+    for (int x = tid - kPredPos * 32; x < kPredPos * kPredHid; x += kTailThreads - kPredPos * 32)
+      sf[kPredPos * kPredConf + x] = hsrc[x];
+    if (warp == kPredPos && lane < kPredCtx)
+      sf[kPredFeatures - kPredCtx + lane] = lane == 0 ? (float)n : (lane == 3 ? 1.f : 0.f);
   }
   __syncthreads();
+  if (m.features_out)
+    for (int x = tid; x < kPredFeatures; x += kTailThreads) m.features_out[(size_t)i * kPredFeatures + x] = sf[x];
   {
     // warp w computes hidden units 2 w and 2 w + 1: many independent weight loads in flight
-    const float* w0 = a.w1 + (size_t)(2 * warp) * kPredFeatures;
+    const float* w0 = m.w1 + (size_t)(2 * warp) * kPredFeatures;
     const float* w1 = w0 + kPredFeatures;
     float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll 8
+#pragma unroll 14
     for (int x = lane; x < kPredFeatures; x += 32) {
       const float fx = sf[x];
       acc0 = fmaf(__ldg(w0 + x), fx, acc0);
@@ -662,17 +693,17 @@ __global__ void __launch_bounds__(kMlpThreads) pred_mlp_kernel(MlpArgs a) {
       acc1 += __shfl_xor_sync(0xffffffffu, acc1, o);
     }
     if (lane == 0) {
-      sh[2 * warp] = fmaxf(acc0 + a.b1[2 * warp], 0.f);
-      sh[2 * warp + 1] = fmaxf(acc1 + a.b1[2 * warp + 1], 0.f);
+      sh[2 * warp] = fmaxf(acc0 + m.b1[2 * warp], 0.f);
+      sh[2 * warp + 1] = fmaxf(acc1 + m.b1[2 * warp + 1], 0.f);
     }
   }
   __syncthreads();
   if (warp < kPredPos) {
-    const float* w = a.w2 + warp * kPredMlp;
+    const float* w = m.w2 + warp * kPredMlp;
     float acc = w[lane] * sh[lane] + w[lane + 32] * sh[lane + 32];
 #pragma unroll
     for (int x = 16; x > 0; x >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, x);
-    if (lane == 0) a.pred_logits[i * kPredPos + warp] = acc + a.b2[warp];
+    if (lane == 0) m.pred_logits[i * kPredPos + warp] = acc + m.b2[warp];
   }
 }
 
@@ -753,7 +784,7 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   // The hidden-state projection does not depend on the logit stream and is small: it goes
   // first and lets its dependents start at once; the stream kernel is launched with
   // programmatic stream serialisation and waits for it only as its last action, so the two
-  // overlap.  The feature merge and the perceptron are ordinary launches behind the
+  // overlap.  The tail kernel (feature merge + perceptron) is launched the same way behind the
   // stream kernel, whose completion then implies the hidden projection's.
   pred_hidden_kernel<<<dim3((kPredPos * p.n_bs + 15) / 16, kHidSlices), kHidThreads, 0, stream>>>(fa);
   cudaError_t e = cudaGetLastError();
@@ -772,12 +803,20 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
     e = cudaLaunchKernelEx(&cfg, pred_stream_kernel, sa, tz, tp);
     if (e != cudaSuccess) return e;
   }
-  pred_features_kernel<<<p.n_bs, kFeatThreads, 0, stream>>>(fa);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
   MlpArgs ma{p.n_live, p.n_bs, feat, p.w1, p.b1, p.w2, p.b2, p.pred_logits, p.features_out};
-  pred_mlp_kernel<<<p.n_bs, kMlpThreads, 0, stream>>>(ma);
-  return cudaGetLastError();
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.n_bs);
+    cfg.blockDim = dim3(kTailThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, pred_tail_kernel, fa, ma);
+  }
+  return e;
 }
 
 }  // namespace dscale
