@@ -558,17 +558,30 @@ struct MlpArgs {
   const float* b2;
   float* pred_logits;   // [n_bs][15]
   float* features_out;  // nullable [n_bs][1735]
+  int* status;          // workspace status word
 };
 
 // ---------------------------------------------------------------------------
 // Per request, behind the stream: merge the chunk records into the 18 confidence values and the
 // centred logit projection of each position, append the hidden-state projection and the batch
-// context, then relu(W1 f + b1) and W2 h + b2.  One launch (the merge and the perceptron used to
-// be two, each paying a launch and a cold pass over its inputs); it is launched with
-// programmatic stream serialisation: everything that depends only on the call's inputs (the
-// pivots, pulling W1 into L2 with an evict-last hint while the logit stream is still running)
-// happens before the grid dependency is waited for.
-constexpr int kTailThreads = 1024;                          // 32 warps: a position each, then two hidden units each
+// context, then relu(W1 f + b1) and W2 h + b2.  A request is served by a cluster of four CTAs:
+// each merges a quarter of the positions and stores its features into the shared memory of all
+// four, and each computes 16 of the 64 hidden units from its own quarter of W1 (111 KB, fetched
+// into shared memory by one bulk copy), so that no single SM has to pull all of W1 through its
+// L2 port; the hidden units meet in the first CTA, which applies W2.  The launch uses
+// programmatic stream serialisation: everything that depends only on the call's inputs (the W1
+// copy, the pivots, the biases) happens before the grid dependency is waited for, while the
+// logit stream is still running.
+constexpr int kTailCtas = 4;                                // CTAs (one cluster) per request
+constexpr int kTailThreads = 512;                           // 16 warps: a hidden unit each
+constexpr int kTailUnits = kPredMlp / kTailCtas;            // hidden units per CTA
+constexpr int kTailW1 = kTailUnits * kPredFeatures;         // floats of W1 per CTA (111,040 bytes)
+constexpr int kTailMergeWarps = (kPredPos + kTailCtas - 1) / kTailCtas;   // positions per CTA
+constexpr int kTailSf = (kPredFeatures + 3) / 4 * 4;
+constexpr int kTailCand = 16 * kPredMaxChunks;              // candidate values of one position
+constexpr int kTailSmem = (kTailW1 + kTailSf + kPredMlp + kTailMergeWarps * kTailCand) * 4 + 32;
+static_assert(kTailUnits * 32 == kTailThreads, "one warp per hidden unit");
+static_assert((kTailW1 * 4) % 16 == 0, "bulk copy size");
 
 // order-preserving key of a float for integer warp reductions; a NaN gets the lowest key
 __device__ __forceinline__ unsigned f2key(float v) {
@@ -578,41 +591,72 @@ __device__ __forceinline__ unsigned f2key(float v) {
 __device__ __forceinline__ float key2f(unsigned k) {
   return __uint_as_float(k ^ ((k >> 31) ? 0x80000000u : 0xffffffffu));
 }
+__device__ __forceinline__ uint32_t tail_cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// store into the same shared-memory variable of another CTA of the cluster
+__device__ __forceinline__ void st_cluster(const float* local, uint32_t rank, float v) {
+  uint32_t addr;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(addr) : "r"(smem_u32(local)), "r"(rank));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void tail_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
-__global__ void __launch_bounds__(kTailThreads, 1) pred_tail_kernel(FeatArgs a, MlpArgs m) {
-  __shared__ float sf[kPredFeatures];
-  __shared__ float sh[kPredMlp];
-  const int i = blockIdx.x;
+__global__ void __cluster_dims__(kTailCtas, 1, 1) __launch_bounds__(kTailThreads, 1)
+pred_tail_kernel(FeatArgs a, MlpArgs m) {
+  extern __shared__ __align__(16) unsigned char tail_smem[];
+  float* w1s = reinterpret_cast<float*>(tail_smem);         // this CTA's 16 rows of W1
+  float* sf = w1s + kTailW1;                                // the request's feature vector
+  float* sh = sf + kTailSf;                                 // hidden units (complete in CTA 0)
+  float* cs = sh + kPredMlp;                                // candidate staging, one array per merging warp
+  const uint32_t bar = smem_u32(cs + kTailMergeWarps * kTailCand);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(cs + kTailMergeWarps * kTailCand + 2);
+  const uint32_t rank = tail_cluster_rank();
+  const int i = blockIdx.x / kTailCtas;
   int n = *a.n_live;
   n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool live = i < n;
+  const bool live = i < n;                                  // the same for the four CTAs of a cluster
+  const bool bulk = (reinterpret_cast<uintptr_t>(m.w1) & 15) == 0;
+  const int unit = kTailUnits * (int)rank + warp;           // this warp's hidden unit
   // ---- before the grid dependency: inputs of the call only
-  float pivot = 0.f;
-  if (live) {
-    for (int x = tid * 32; x < kPredMlp * kPredFeatures; x += kTailThreads * 32)
-      asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(m.w1 + x));
-    if (warp < kPredPos) pivot = a.logits[(size_t)(i * kPredPos + warp) * a.ld];
+  if (tid == 0) {
+    mbar_init(bar, 1);
+    s_abort[0] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (live && bulk) {
+      mbar_expect_tx(bar, kTailW1 * 4);
+      bulk_load(smem_u32(w1s), m.w1 + (size_t)rank * kTailW1, kTailW1 * 4, bar);
+    }
   }
+  const int p = (int)rank + kTailCtas * warp;               // the position a merging warp serves
+  const bool merges = warp < kTailMergeWarps && p < kPredPos;
+  float pivot = 0.f, b1v = 0.f;
+  if (live) {
+    if (merges) pivot = a.logits[(size_t)(i * kPredPos + p) * a.ld];
+    b1v = m.b1[unit];
+  }
+  __syncthreads();                                          // the barrier is initialised for every waiter
   pdl_wait();
-  if (!live) {                                              // dead request: zeros
-    if (tid < kPredPos) m.pred_logits[i * kPredPos + tid] = 0.f;
-    if (m.features_out)
-      for (int x = tid; x < kPredFeatures; x += kTailThreads) m.features_out[(size_t)i * kPredFeatures + x] = 0.f;
+  if (!live) {                                              // dead request: zeros (the whole cluster leaves)
+    if (rank == 0) {
+      if (tid < kPredPos) m.pred_logits[i * kPredPos + tid] = 0.f;
+      if (m.features_out)
+        for (int x = tid; x < kPredFeatures; x += kTailThreads) m.features_out[(size_t)i * kPredFeatures + x] = 0.f;
+    }
     return;
   }
-  if (warp < kPredPos) {
-    // ---- confidence values and centred logit projection, one warp per position
-    const int p = warp;
+  if (merges) {
+    // ---- confidence values and centred logit projection of position p
     const int row = i * kPredPos + p;
     const float* rec0 = a.part + (size_t)row * a.chunks * kPredRec;
+    float* cw = cs + warp * kTailCand;
     // all loads of this position first (independent), then the merges
-    unsigned cand[kPredMaxChunks / 2];                      // lane l: candidate l % 16 of chunk 2 x + l / 16
-#pragma unroll
-    for (int x = 0; x < kPredMaxChunks / 2; ++x) {
-      const int c = 2 * x + (lane >> 4);
-      cand[x] = c < a.chunks ? f2key(rec0[(size_t)c * kPredRec + (lane & 15)]) : 0u;
-    }
+    for (int e = lane; e < 16 * a.chunks; e += 32) cw[e] = rec0[(size_t)(e >> 4) * kPredRec + (e & 15)];
     float proj = 0.f, rs = 0.f;
 #pragma unroll 8
     for (int c = 0; c < a.chunks; ++c) {
@@ -624,22 +668,20 @@ __global__ void __launch_bounds__(kTailThreads, 1) pred_tail_kernel(FeatArgs a, 
       const float* r = rec0 + (size_t)lane * kPredRec;
       mx = r[16]; s_sum = r[17]; t_sum = r[18]; z_sum = r[19];
     }
-    // the 16 largest of all chunks' candidates, in order: sixteen rounds of (lane maximum, warp
-    // maximum by an integer reduction, the first lane holding it gives it up)
+    __syncwarp();
+    // The 16 largest of all chunks' candidates, in order.  Every chunk's list is sorted, so
+    // this is a merge: lane c holds the head of chunk c, the warp maximum (an integer
+    // reduction on order-preserving keys) is the next value, the first lane holding it advances.
     float tv = -INFINITY;                                   // lane j < 16: the (j + 1)-th largest
+    int ptr = 0;
+    unsigned head = lane < a.chunks ? f2key(cw[16 * lane]) : 0u;
 #pragma unroll 1
     for (int j = 0; j < 16; ++j) {
-      unsigned lm = 0u;
-#pragma unroll
-      for (int x = 0; x < kPredMaxChunks / 2; ++x)
-        if (2 * x < a.chunks) lm = max(lm, cand[x]);
-      const unsigned gm = __reduce_max_sync(0xffffffffu, lm);
-      const unsigned who = __ballot_sync(0xffffffffu, lm == gm);
+      const unsigned gm = __reduce_max_sync(0xffffffffu, head);
+      const unsigned who = __ballot_sync(0xffffffffu, head == gm);
       if (lane == __ffs(who) - 1) {
-        bool gone = false;
-#pragma unroll
-        for (int x = 0; x < kPredMaxChunks / 2; ++x)
-          if (2 * x < a.chunks && !gone && cand[x] == gm) { cand[x] = 0u; gone = true; }
+        ++ptr;
+        head = (lane < a.chunks && ptr < 16) ? f2key(cw[16 * lane + ptr]) : 0u;
       }
       if (lane == j) tv = gm != 0u ? key2f(gm) : -INFINITY;
     }
@@ -657,48 +699,49 @@ __global__ void __launch_bounds__(kTailThreads, 1) pred_tail_kernel(FeatArgs a, 
     }
     const float lse = mx + logf(s_sum);
     const float top = __shfl_sync(0xffffffffu, tv, 0);
-    float* fc = sf + p * kPredConf;
-    if (lane == 0) fc[0] = top;
-    else if (lane < 16) fc[lane] = top - tv;
-    else if (lane == 16) fc[16] = top - lse;
-    else if (lane == 17) fc[17] = lse - t_sum / s_sum;
+    float conf = 0.f;
+    if (lane == 0) conf = top;
+    else if (lane < 16) conf = top - tv;
+    else if (lane == 16) conf = top - lse;
+    else if (lane == 17) conf = lse - t_sum / s_sum;
     // logit projection of z - mean(z): the stream accumulated P (z - pivot)
     const float mean = z_sum / (float)a.vocab;
-    sf[kPredPos * (kPredConf + kPredHid) + p * kPredLog + lane] = proj - (mean - pivot) * rs;
-  } else {
+    const float cproj = proj - (mean - pivot) * rs;
+#pragma unroll
+    for (uint32_t dst = 0; dst < kTailCtas; ++dst) {
+      if (lane < kPredConf) st_cluster(sf + p * kPredConf + lane, dst, conf);
+      st_cluster(sf + kPredPos * (kPredConf + kPredHid) + p * kPredLog + lane, dst, cproj);
+    }
+  } else if (warp >= kTailMergeWarps) {
     // ---- the other warps: the hidden-state projection of this request and the batch context
+    constexpr int kRest = kTailThreads - kTailMergeWarps * 32;
     const float* hsrc = a.feat + (size_t)i * kPredFeatures + kPredPos * kPredConf;
-    for (int x = tid - kPredPos * 32; x < kPredPos * kPredHid; x += kTailThreads - kPredPos * 32)
-      sf[kPredPos * kPredConf + x] = hsrc[x];
-    if (warp == kPredPos && lane < kPredCtx)
+    for (int x = tid - kTailMergeWarps * 32; x < kPredPos * kPredHid; x += kRest) sf[kPredPos * kPredConf + x] = hsrc[x];
+    if (warp == kTailMergeWarps && lane < kPredCtx)
       sf[kPredFeatures - kPredCtx + lane] = lane == 0 ? (float)n : (lane == 3 ? 1.f : 0.f);
   }
-  __syncthreads();
-  if (m.features_out)
+  tail_cluster_sync();                                      // the feature vector is complete in all four CTAs
+  if (rank == 0 && m.features_out)
     for (int x = tid; x < kPredFeatures; x += kTailThreads) m.features_out[(size_t)i * kPredFeatures + x] = sf[x];
   {
-    // warp w computes hidden units 2 w and 2 w + 1: many independent weight loads in flight
-    const float* w0 = m.w1 + (size_t)(2 * warp) * kPredFeatures;
-    const float* w1 = w0 + kPredFeatures;
-    float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll 14
-    for (int x = lane; x < kPredFeatures; x += 32) {
-      const float fx = sf[x];
-      acc0 = fmaf(__ldg(w0 + x), fx, acc0);
-      acc1 = fmaf(__ldg(w1 + x), fx, acc1);
-    }
+    // ---- warp w: hidden unit 16 rank + w from this CTA's rows of W1
+    bool have = bulk && mbar_wait(bar, 0, s_abort);
+    const float* wrow = have ? w1s + warp * kPredFeatures : m.w1 + (size_t)unit * kPredFeatures;
+    float acc = 0.f;
+#pragma unroll 8
+    for (int x = lane; x < kPredFeatures; x += 32) acc = fmaf(wrow[x], sf[x], acc);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      acc0 += __shfl_xor_sync(0xffffffffu, acc0, o);
-      acc1 += __shfl_xor_sync(0xffffffffu, acc1, o);
-    }
-    if (lane == 0) {
-      sh[2 * warp] = fmaxf(acc0 + m.b1[2 * warp], 0.f);
-      sh[2 * warp + 1] = fmaxf(acc1 + m.b1[2 * warp + 1], 0.f);
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) st_cluster(sh + unit, 0, fmaxf(acc + b1v, 0.f));
+    if (bulk && !have) {
+      // the copy did not land within the limit: flag it, and do not leave while it may still be writing
+      if (lane == 0) atomicOr(m.status, 8 /*TIMEOUT*/);
+      volatile int again = 0;
+      mbar_wait(bar, 0, &again);
     }
   }
-  __syncthreads();
-  if (warp < kPredPos) {
+  tail_cluster_sync();                                      // all 64 hidden units are in CTA 0
+  if (rank == 0 && warp < kPredPos) {
     const float* w = m.w2 + warp * kPredMlp;
     float acc = w[lane] * sh[lane] + w[lane + 32] * sh[lane + 32];
 #pragma unroll
@@ -741,7 +784,9 @@ static bool pred_encode(CUtensorMap* out, CUtensorMapDataType dt, const void* pt
 }
 
 cudaError_t predictor_prepare() {
-  return cudaFuncSetAttribute(pred_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
+  cudaError_t e = cudaFuncSetAttribute(pred_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(pred_tail_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTailSmem);
 }
 
 int predictor_chunks(int n_bs, int vocab, int num_ctas, int* chunk_len_out) {
@@ -803,11 +848,13 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
     e = cudaLaunchKernelEx(&cfg, pred_stream_kernel, sa, tz, tp);
     if (e != cudaSuccess) return e;
   }
-  MlpArgs ma{p.n_live, p.n_bs, feat, p.w1, p.b1, p.w2, p.b2, p.pred_logits, p.features_out};
+  MlpArgs ma{p.n_live, p.n_bs, feat, p.w1, p.b1, p.w2, p.b2, p.pred_logits, p.features_out,
+             ws_ptr<int>(p.ws, L.hdr) + H_STATUS};
   {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.n_bs);
+    cfg.gridDim = dim3(kTailCtas * p.n_bs);
     cfg.blockDim = dim3(kTailThreads);
+    cfg.dynamicSmemBytes = kTailSmem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
