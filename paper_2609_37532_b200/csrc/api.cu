@@ -446,7 +446,7 @@ int dscale_launches_per_call(int which) {
     case 4: return 1;   // attn_padded_kernel
     case 5: return 2;   // sample_stats_kernel + sample_draw_kernel
     case 6: return 1;   // lm_head_kernel
-    case 7: return 3;   // pred_hidden_kernel, pred_stream_kernel, pred_tail_kernel
+    case 7: return 2;   // pred_stream_kernel, pred_tail_kernel
     default: return 0;
   }
 }

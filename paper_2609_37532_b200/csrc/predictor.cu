@@ -1,7 +1,6 @@
 // Acceptance-predictor front end: drafter logits and hidden states -> 1735
 // features -> 1735-64-15 perceptron -> predLogits ("Acceptance predictor"
-// paragraph, Eq. 4 and Eq. 5).  Three launches (the hidden-state projection goes first and
-// overlaps with the logit stream; the tail is scheduled while the stream runs):
+// paragraph, Eq. 4 and Eq. 5).  Two launches (the tail is scheduled while the stream runs):
 //
 //  pred_stream_kernel    the only pass over the drafter logits (15 N rows x V fp32,
 //                        292 MB at N = 32: an HBM stream).  A CTA of 16 warps owns
@@ -20,7 +19,9 @@
 //                        along with a 292 MB stream, there is no tensor-core
 //                        time to win, and the rows are already in registers.
 //                        One record per (row, chunk) goes to the workspace.
-//  pred_hidden_kernel    the 64 x H hidden-state projection of all rows (bf16 MMAs).
+//                        The CTAs of the grid behind the (row group, chunk) CTAs compute
+//                        the 64 x H hidden-state projection of all rows (bf16 MMAs) on
+//                        the SMs the stream leaves free.
 //  pred_tail_kernel      per request: merges the chunk records into the 18
 //                        confidence values and the centred logit projection per
 //                        position, appends the hidden projection and the batch
@@ -50,11 +51,19 @@ struct StreamArgs {
   int n_bs;
   const __nv_bfloat16* p_logit;   // [32][vocab]
   float* part;              // [15 n_bs][chunks][kPredRec]
-  float* rowsum;            // [chunks][32]
+  float* rowsum;            // [row groups][chunks][32]: partial row sums of the projection matrix
   int chunks;
   int chunk_len;            // multiple of kSub
+  int stream_ctas;          // chunks x row groups; the CTAs behind them serve the hidden projection
   int* status;              // workspace status word
+  const __nv_bfloat16* hidden;     // [n_bs][15][hidden_dim]
+  int hidden_dim;
+  const __nv_bfloat16* p_hidden;   // [64][hidden_dim]
+  float* feat;                     // [n_bs][1735]
 };
+constexpr int kHidThreads = 256;                // threads of one hidden-projection job
+constexpr int kHidJobs = kWarps * 32 / kHidThreads;   // jobs side by side in a CTA that serves them
+constexpr int kHidSlices = 4;                   // 16 of the 64 outputs per job
 
 __device__ __forceinline__ float to_tf32(float x) {
   uint32_t r;
@@ -226,6 +235,81 @@ __device__ __forceinline__ void row_update2(RowStat& a, RowStat& b, float4 za, f
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// ---------------------------------------------------------------------------
+// Hidden-state projection: [15 N rows x H] . [H x 64], a small dense contraction
+// (0.25 GFLOP at N = 32, H = 4096) on warp-level bf16 MMAs.  It does not depend on the
+// logit stream: the CTAs of the stream grid that are left over once every (row group,
+// chunk) has its CTA serve it, two jobs of 256 threads side by side, while the stream runs
+// on the other SMs.  (As a kernel of its own ahead of the stream it held the stream's CTAs
+// off its SMs for the 10 us it ran: the two did not share an SM.)  A job owns 16 rows x 16
+// outputs; its 8 warps split H in blocks of 32 and are summed through shared memory.  The
+// k slots of the MMA are a permutation of the 32 columns of a block (the same one for both
+// operands), so every fragment is one 16-byte load.
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void job_barrier(int job) {
+  asm volatile("bar.sync %0, %1;" ::"r"(job + 1), "r"(kHidThreads) : "memory");
+}
+__device__ void hidden_jobs(const StreamArgs& a, int live_rows, int first_item, int item_stride, int job,
+                            int tid /* within the job */, float* red /* [8][256] */) {
+  constexpr int kOut = kPredHid / kHidSlices;               // 16 outputs = 2 n-tiles
+  const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int H = a.hidden_dim;
+  const int row_tiles = (live_rows + 15) / 16;
+  for (int item = first_item; item < row_tiles * kHidSlices; item += item_stride) {
+    const int row0 = (item / kHidSlices) * 16, j0 = (item % kHidSlices) * kOut;
+    const int r_lo = min(row0 + g, live_rows - 1), r_hi = min(row0 + g + 8, live_rows - 1);
+    const __nv_bfloat16* h_lo = a.hidden + (size_t)r_lo * H;
+    const __nv_bfloat16* h_hi = a.hidden + (size_t)r_hi * H;
+    const __nv_bfloat16* p0 = a.p_hidden + (size_t)(j0 + g) * H;
+    const __nv_bfloat16* p1 = a.p_hidden + (size_t)(j0 + 8 + g) * H;
+    float d[2][4];
+#pragma unroll
+    for (int x = 0; x < 2; ++x) d[x][0] = d[x][1] = d[x][2] = d[x][3] = 0.f;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    constexpr int kStep = 32 * (kHidThreads / 32);          // columns per round of the 8 warps
+#pragma unroll 4
+    for (int kb = warp * 32; kb < H; kb += kStep) {
+      const int c = kb + 8 * t;                            // hidden_dim % 8 == 0: a chunk is in or out
+      const bool in = c < H;
+      const uint4 alo = in ? __ldg(reinterpret_cast<const uint4*>(h_lo + c)) : zero4;
+      const uint4 ahi = in ? __ldg(reinterpret_cast<const uint4*>(h_hi + c)) : zero4;
+      const uint4 b0 = in ? __ldg(reinterpret_cast<const uint4*>(p0 + c)) : zero4;
+      const uint4 b1 = in ? __ldg(reinterpret_cast<const uint4*>(p1 + c)) : zero4;
+      mma_bf16(d[0], alo.x, ahi.x, alo.y, ahi.y, b0.x, b0.y);
+      mma_bf16(d[0], alo.z, ahi.z, alo.w, ahi.w, b0.z, b0.w);
+      mma_bf16(d[1], alo.x, ahi.x, alo.y, ahi.y, b1.x, b1.y);
+      mma_bf16(d[1], alo.z, ahi.z, alo.w, ahi.w, b1.z, b1.w);
+    }
+    float* rw = red + warp * (16 * kOut);
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+      rw[g * kOut + 8 * nt + 2 * t] = d[nt][0];
+      rw[g * kOut + 8 * nt + 2 * t + 1] = d[nt][1];
+      rw[(g + 8) * kOut + 8 * nt + 2 * t] = d[nt][2];
+      rw[(g + 8) * kOut + 8 * nt + 2 * t + 1] = d[nt][3];
+    }
+    job_barrier(job);
+    {
+      const int x = tid;                                    // 16 rows x 16 outputs = 256 = kHidThreads
+      float acc = 0.f;
+#pragma unroll
+      for (int w = 0; w < kHidThreads / 32; ++w) acc += red[w * (16 * kOut) + x];
+      const int row = row0 + (x >> 4), j = j0 + (x & 15);
+      if (row < live_rows) {
+        const int i = row / kPredPos, p = row - i * kPredPos;
+        a.feat[(size_t)i * kPredFeatures + kPredPos * kPredConf + p * kPredHid + j] = acc;
+      }
+    }
+    job_barrier(job);                                       // the buffer is free for the next item
+  }
+}
+
 __global__ void __launch_bounds__(kStreamThreads, 1)
 pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const __grid_constant__ CUtensorMap tm_p) {
   extern __shared__ unsigned char smem_raw[];
@@ -247,18 +331,33 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
   int n = *a.n_live;
   n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
   const int live_rows = kPredPos * n;
-  const int row0 = blockIdx.y * kRowsPerCta;
-  if (row0 >= live_rows) { pdl_wait(); return; }
-  const int chunk = blockIdx.x;
+  if ((int)blockIdx.x >= a.stream_ctas) {
+    // ===================================================== hidden-state projection
+    if (warp < kHidJobs * (kHidThreads / 32) && live_rows > 0) {
+      const int job = tid / kHidThreads;
+      hidden_jobs(a, live_rows, ((int)blockIdx.x - a.stream_ctas) * kHidJobs + job,
+                  ((int)gridDim.x - a.stream_ctas) * kHidJobs, job, tid - job * kHidThreads,
+                  reinterpret_cast<float*>(smem) + job * (kHidThreads / 32) * 256);
+    }
+    return;
+  }
+  const int row_group = (int)blockIdx.x / a.chunks;
+  const int row0 = row_group * kRowsPerCta;
+  if (row0 >= live_rows) return;
+  const int chunk = (int)blockIdx.x % a.chunks;
   const int col_lo = chunk * a.chunk_len;
   const int col_hi = min(a.vocab, col_lo + a.chunk_len);
-  if (col_lo >= col_hi) { pdl_wait(); return; }
+  if (col_lo >= col_hi) return;
   const int n_sub = (col_hi - col_lo + kSub - 1) / kSub;
 
   // warp w owns rows w and w + 16 of the CTA's 32 (one in each 16-row MMA tile)
   const int my_row[2] = {row0 + warp, row0 + warp + kWarps};
   const bool live[2] = {warp < kWarps && my_row[0] < live_rows, warp < kWarps && my_row[1] < live_rows};
   const bool p_vec = (a.vocab & 7) == 0;               // projection rows 16-byte aligned
+  // The centring term of the logit projection needs the row sums of the projection matrix.  Its
+  // tiles pass through the shared memory of every row group's CTAs; the live row groups take
+  // turns by sub-tile, so each CTA sums a share of its chunk and none is slower than the others.
+  const int live_groups = (live_rows + kRowsPerCta - 1) / kRowsPerCta;
   const int pj = tid >> 4, pq = tid & 15;               // projection tile piece: (output, 8 columns)
 
   if (tid == 0) {
@@ -343,6 +442,7 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
   const uint32_t po = kOffP + p_off(g, 8 * (warp & 15) + 2 * t);    // + 1024 per output tile
   const uint32_t so0 = z_off(warp & 15, 4 * lane), so1 = z_off((warp & 15) + kWarps, 4 * lane);
   const uint32_t ro = kOffP + p_off(pj & 31, 8 * pq);               // row sums: eight weights of output pj
+  int rs_turn = row_group;                                          // sub-tiles until this CTA's turn
 
   int st = 0;
   uint32_t parity = 0;
@@ -376,14 +476,16 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
         for (int nt = 0; nt < 4; ++nt) mma_tf32(d[h][nt], af, bw[nt] << 16, bw[nt] & 0xffff0000u);
       }
     }
-    // ---- row sums of the projection matrix (first row group only)
-    if (blockIdx.y == 0) {
+    // ---- row sums of the projection matrix (this row group's turn)
+    if (rs_turn == 0) {
+      rs_turn = live_groups;
       const uint4 w = *reinterpret_cast<const uint4*>(pst + ro);
       const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
       for (int x = 0; x < 4; ++x)
         p_rowsum += __uint_as_float(ww[x] << 16) + __uint_as_float(ww[x] & 0xffff0000u);
     }
+    --rs_turn;
     __syncwarp();
     if (lane == 0) mbar_arrive(empty(st));                  // this warp is done with the stage
     if (++st == kStages) { st = 0; parity ^= 1; }
@@ -393,8 +495,6 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
     // Some wait ran out (the copy warp has already waited for its copies): flag the
     // status word and leave.
     if (tid == 0) atomicOr(a.status, 8 /*TIMEOUT*/);
-    __syncthreads();
-    pdl_wait();
     return;
   }
 
@@ -444,17 +544,11 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
     if (row0 + r < live_rows)
       a.part[((size_t)(row0 + r) * a.chunks + chunk) * kPredRec + 20 + j] = acc;
   }
-  if (blockIdx.y == 0 && warp < kWarps) {
+  if (warp < kWarps) {
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) p_rowsum += __shfl_xor_sync(0xffffffffu, p_rowsum, o);
-    if (pq == 0) a.rowsum[chunk * kPredLog + pj] = p_rowsum;
+    if (pq == 0) a.rowsum[((size_t)row_group * a.chunks + chunk) * kPredLog + pj] = p_rowsum;
   }
-  // This grid was allowed to start before the hidden-projection kernel ahead of it in
-  // the stream had finished (it reads nothing that kernel writes).  The kernels behind
-  // this one do read it, and they are ordered only behind this grid: waiting here, as
-  // the last thing every CTA does, makes this grid's completion imply the completion
-  // and memory flush of that kernel.
-  pdl_wait();
 }
 
 // ---------------------------------------------------------------------------
@@ -472,80 +566,6 @@ struct FeatArgs {
   int chunks;
   float* feat;                     // [n_bs][1735]
 };
-
-// ---------------------------------------------------------------------------
-// Hidden-state projection: [15 N rows x H] . [H x 64], a small dense contraction
-// (0.25 GFLOP at N = 32, H = 4096) on warp-level bf16 MMAs.  A CTA owns 16 rows;
-// its 8 warps split H in blocks of 32 and are summed through shared memory.  The
-// k slots of the MMA are a permutation of the 32 columns of a block (the same
-// one for both operands), so every fragment is one 16-byte load.
-constexpr int kHidThreads = 256;
-
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-constexpr int kHidSlices = 4;                               // grid.y: 16 of the 64 outputs each
-
-__global__ void __launch_bounds__(kHidThreads) pred_hidden_kernel(FeatArgs a) {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the logit stream may start now
-  constexpr int kOut = kPredHid / kHidSlices;               // 16 outputs = 2 n-tiles
-  __shared__ float red[kHidThreads / 32][16 * kOut];
-  int n = *a.n_live;
-  n = n < 0 ? 0 : (n > a.n_bs ? a.n_bs : n);
-  const int live_rows = kPredPos * n;
-  const int row0 = blockIdx.x * 16;
-  if (row0 >= live_rows) return;
-  const int j0 = blockIdx.y * kOut;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int H = a.hidden_dim;
-  const int r_lo = min(row0 + g, live_rows - 1), r_hi = min(row0 + g + 8, live_rows - 1);
-  const __nv_bfloat16* h_lo = a.hidden + (size_t)r_lo * H;
-  const __nv_bfloat16* h_hi = a.hidden + (size_t)r_hi * H;
-  const __nv_bfloat16* p0 = a.p_hidden + (size_t)(j0 + g) * H;
-  const __nv_bfloat16* p1 = a.p_hidden + (size_t)(j0 + 8 + g) * H;
-  float d[2][4];
-#pragma unroll
-  for (int x = 0; x < 2; ++x) d[x][0] = d[x][1] = d[x][2] = d[x][3] = 0.f;
-  const uint4 zero4 = make_uint4(0, 0, 0, 0);
-  constexpr int kStep = 32 * (kHidThreads / 32);            // columns per round of the 8 warps
-#pragma unroll 4
-  for (int kb = warp * 32; kb < H; kb += kStep) {
-    const int c = kb + 8 * t;                              // hidden_dim % 8 == 0: a chunk is in or out
-    const bool in = c < H;
-    const uint4 alo = in ? __ldg(reinterpret_cast<const uint4*>(h_lo + c)) : zero4;
-    const uint4 ahi = in ? __ldg(reinterpret_cast<const uint4*>(h_hi + c)) : zero4;
-    const uint4 b0 = in ? __ldg(reinterpret_cast<const uint4*>(p0 + c)) : zero4;
-    const uint4 b1 = in ? __ldg(reinterpret_cast<const uint4*>(p1 + c)) : zero4;
-    mma_bf16(d[0], alo.x, ahi.x, alo.y, ahi.y, b0.x, b0.y);
-    mma_bf16(d[0], alo.z, ahi.z, alo.w, ahi.w, b0.z, b0.w);
-    mma_bf16(d[1], alo.x, ahi.x, alo.y, ahi.y, b1.x, b1.y);
-    mma_bf16(d[1], alo.z, ahi.z, alo.w, ahi.w, b1.z, b1.w);
-  }
-#pragma unroll
-  for (int nt = 0; nt < 2; ++nt) {
-    red[warp][g * kOut + 8 * nt + 2 * t] = d[nt][0];
-    red[warp][g * kOut + 8 * nt + 2 * t + 1] = d[nt][1];
-    red[warp][(g + 8) * kOut + 8 * nt + 2 * t] = d[nt][2];
-    red[warp][(g + 8) * kOut + 8 * nt + 2 * t + 1] = d[nt][3];
-  }
-  __syncthreads();
-  {
-    const int x = tid;                                      // 16 rows x 16 outputs = 256 = kHidThreads
-    float acc = 0.f;
-#pragma unroll
-    for (int w = 0; w < kHidThreads / 32; ++w) acc += red[w][x];
-    const int row = row0 + (x >> 4), j = j0 + (x & 15);
-    if (row < live_rows) {
-      const int i = row / kPredPos, p = row - i * kPredPos;
-      a.feat[(size_t)i * kPredFeatures + kPredPos * kPredConf + p * kPredHid + j] = acc;
-    }
-  }
-}
 
 // ---------------------------------------------------------------------------
 struct MlpArgs {
@@ -579,7 +599,8 @@ constexpr int kTailW1 = kTailUnits * kPredFeatures;         // floats of W1 per 
 constexpr int kTailMergeWarps = (kPredPos + kTailCtas - 1) / kTailCtas;   // positions per CTA
 constexpr int kTailSf = (kPredFeatures + 3) / 4 * 4;
 constexpr int kTailCand = 16 * kPredMaxChunks;              // candidate values of one position
-constexpr int kTailSmem = (kTailW1 + kTailSf + kPredMlp + kTailMergeWarps * kTailCand) * 4 + 32;
+constexpr int kTailRest = kTailThreads / 32 - kTailMergeWarps;    // warps that do not merge a position
+constexpr int kTailSmem = (kTailW1 + kTailSf + kPredMlp + kTailRest * kPredLog + kTailMergeWarps * kTailCand) * 4 + 32;
 static_assert(kTailUnits * 32 == kTailThreads, "one warp per hidden unit");
 static_assert((kTailW1 * 4) % 16 == 0, "bulk copy size");
 
@@ -612,7 +633,8 @@ pred_tail_kernel(FeatArgs a, MlpArgs m) {
   float* w1s = reinterpret_cast<float*>(tail_smem);         // this CTA's 16 rows of W1
   float* sf = w1s + kTailW1;                                // the request's feature vector
   float* sh = sf + kTailSf;                                 // hidden units (complete in CTA 0)
-  float* cs = sh + kPredMlp;                                // candidate staging, one array per merging warp
+  float* rsp = sh + kPredMlp;                               // partial row sums of the projection matrix, one array per non-merging warp
+  float* cs = rsp + kTailRest * kPredLog;                   // candidate staging, one array per merging warp
   const uint32_t bar = smem_u32(cs + kTailMergeWarps * kTailCand);
   volatile int* s_abort = reinterpret_cast<volatile int*>(cs + kTailMergeWarps * kTailCand + 2);
   const uint32_t rank = tail_cluster_rank();
@@ -650,6 +672,7 @@ pred_tail_kernel(FeatArgs a, MlpArgs m) {
     }
     return;
   }
+  float centre = 0.f, craw = 0.f;                           // mean(z) - pivot and P (z - pivot) of a merging warp's position
   if (merges) {
     // ---- confidence values and centred logit projection of position p
     const int row = i * kPredPos + p;
@@ -657,12 +680,9 @@ pred_tail_kernel(FeatArgs a, MlpArgs m) {
     float* cw = cs + warp * kTailCand;
     // all loads of this position first (independent), then the merges
     for (int e = lane; e < 16 * a.chunks; e += 32) cw[e] = rec0[(size_t)(e >> 4) * kPredRec + (e & 15)];
-    float proj = 0.f, rs = 0.f;
+    float proj = 0.f;
 #pragma unroll 8
-    for (int c = 0; c < a.chunks; ++c) {
-      proj += rec0[(size_t)c * kPredRec + 20 + lane];
-      rs += a.rowsum[c * kPredLog + lane];
-    }
+    for (int c = 0; c < a.chunks; ++c) proj += rec0[(size_t)c * kPredRec + 20 + lane];
     float mx = -INFINITY, s_sum = 0.f, t_sum = 0.f, z_sum = 0.f;   // the chunks' (max, sum, sum e z, sum z): lane = chunk
     if (lane < a.chunks) {
       const float* r = rec0 + (size_t)lane * kPredRec;
@@ -706,19 +726,35 @@ pred_tail_kernel(FeatArgs a, MlpArgs m) {
     else if (lane == 17) conf = lse - t_sum / s_sum;
     // logit projection of z - mean(z): the stream accumulated P (z - pivot)
     const float mean = z_sum / (float)a.vocab;
-    const float cproj = proj - (mean - pivot) * rs;
+    centre = mean - pivot;
+    craw = proj;
 #pragma unroll
-    for (uint32_t dst = 0; dst < kTailCtas; ++dst) {
+    for (uint32_t dst = 0; dst < kTailCtas; ++dst)
       if (lane < kPredConf) st_cluster(sf + p * kPredConf + lane, dst, conf);
-      st_cluster(sf + kPredPos * (kPredConf + kPredHid) + p * kPredLog + lane, dst, cproj);
-    }
   } else if (warp >= kTailMergeWarps) {
-    // ---- the other warps: the hidden-state projection of this request and the batch context
-    constexpr int kRest = kTailThreads - kTailMergeWarps * 32;
+    // ---- the other warps: the row sums of the projection matrix (the stream's CTAs left one
+    // partial vector per live row group and chunk; lane = output, a fixed order of summation),
+    // the hidden-state projection of this request and the batch context
+    const int slots = (kPredPos * n + kRowsPerCta - 1) / kRowsPerCta * a.chunks;
+    float rs = 0.f;
+#pragma unroll 4
+    for (int x = warp - kTailMergeWarps; x < slots; x += kTailRest) rs += a.rowsum[(size_t)x * kPredLog + lane];
+    rsp[(warp - kTailMergeWarps) * kPredLog + lane] = rs;
+    constexpr int kRest = kTailRest * 32;
     const float* hsrc = a.feat + (size_t)i * kPredFeatures + kPredPos * kPredConf;
     for (int x = tid - kTailMergeWarps * 32; x < kPredPos * kPredHid; x += kRest) sf[kPredPos * kPredConf + x] = hsrc[x];
     if (warp == kTailMergeWarps && lane < kPredCtx)
       sf[kPredFeatures - kPredCtx + lane] = lane == 0 ? (float)n : (lane == 3 ? 1.f : 0.f);
+  }
+  __syncthreads();
+  if (merges) {
+    float rs = 0.f;
+#pragma unroll
+    for (int x = 0; x < kTailRest; ++x) rs += rsp[x * kPredLog + lane];
+    const float cproj = craw - centre * rs;
+#pragma unroll
+    for (uint32_t dst = 0; dst < kTailCtas; ++dst)
+      st_cluster(sf + kPredPos * (kPredConf + kPredHid) + p * kPredLog + lane, dst, cproj);
   }
   tail_cluster_sync();                                      // the feature vector is complete in all four CTAs
   if (rank == 0 && m.features_out)
@@ -791,7 +827,9 @@ cudaError_t predictor_prepare() {
 
 int predictor_chunks(int n_bs, int vocab, int num_ctas, int* chunk_len_out) {
   const int row_groups = (kPredPos * n_bs + kRowsPerCta - 1) / kRowsPerCta;
-  int chunks = num_ctas / row_groups;                             // one CTA per SM, a single wave
+  // one CTA per SM, a single wave; about one SM in sixteen is left to the hidden-state projection
+  const int spare = num_ctas / 16 > 1 ? num_ctas / 16 : 1;
+  int chunks = (num_ctas - spare) / row_groups;
   chunks = chunks < 1 ? 1 : (chunks > kPredMaxChunks ? kPredMaxChunks : chunks);
   int chunk_len = (vocab + chunks - 1) / chunks;
   chunk_len = (chunk_len + kSub - 1) / kSub * kSub;
@@ -809,9 +847,17 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   float* feat = ws_ptr<float>(p.ws, L.pred_feat);
   const int row_groups = (kPredPos * p.n_bs + kRowsPerCta - 1) / kRowsPerCta;
 
+  const int stream_ctas = chunks * row_groups;
+  // the hidden-state projection: the SMs the stream leaves free, but no more CTAs than jobs
+  const int hid_items = (kPredPos * p.n_bs + 15) / 16 * kHidSlices;
+  int hid_ctas = p.num_ctas - stream_ctas;
+  hid_ctas = hid_ctas < 1 ? 1 : hid_ctas;
+  hid_ctas = hid_ctas > (hid_items + kHidJobs - 1) / kHidJobs ? (hid_items + kHidJobs - 1) / kHidJobs : hid_ctas;
   StreamArgs sa{p.draft_logits, p.ld, p.vocab, p.n_live, p.n_bs,
                 reinterpret_cast<const __nv_bfloat16*>(p.p_logit), part, rowsum, chunks, chunk_len,
-                ws_ptr<int>(p.ws, L.hdr) + H_STATUS};
+                stream_ctas, ws_ptr<int>(p.ws, L.hdr) + H_STATUS,
+                reinterpret_cast<const __nv_bfloat16*>(p.draft_hidden), p.hidden_dim,
+                reinterpret_cast<const __nv_bfloat16*>(p.p_hidden), feat};
   CUtensorMap tz, tp;
   if (!pred_encode(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, p.draft_logits, (uint64_t)p.vocab,
                    (uint64_t)kPredPos * p.n_bs, (uint64_t)p.ld * 4, 32, kRowsPerCta))
@@ -826,28 +872,13 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   FeatArgs fa{p.draft_logits, p.ld, p.vocab, p.n_live, p.n_bs,
               reinterpret_cast<const __nv_bfloat16*>(p.draft_hidden), p.hidden_dim,
               reinterpret_cast<const __nv_bfloat16*>(p.p_hidden), part, rowsum, chunks, feat};
-  // The hidden-state projection does not depend on the logit stream and is small: it goes
-  // first and lets its dependents start at once; the stream kernel is launched with
-  // programmatic stream serialisation and waits for it only as its last action, so the two
-  // overlap.  The tail kernel (feature merge + perceptron) is launched the same way behind the
-  // stream kernel, whose completion then implies the hidden projection's.
-  pred_hidden_kernel<<<dim3((kPredPos * p.n_bs + 15) / 16, kHidSlices), kHidThreads, 0, stream>>>(fa);
+  // Two launches.  The stream grid carries the hidden-state projection on the CTAs behind its
+  // (row group, chunk) CTAs; the tail kernel (feature merge + perceptron) is launched with
+  // programmatic stream serialisation and does everything that depends only on the call's
+  // inputs while the stream is still running.
+  pred_stream_kernel<<<dim3(stream_ctas + hid_ctas), kStreamThreads, kStreamSmem, stream>>>(sa, tz, tp);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(chunks, row_groups);
-    cfg.blockDim = dim3(kStreamThreads);
-    cfg.dynamicSmemBytes = kStreamSmem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, pred_stream_kernel, sa, tz, tp);
-    if (e != cudaSuccess) return e;
-  }
   MlpArgs ma{p.n_live, p.n_bs, feat, p.w1, p.b1, p.w2, p.b2, p.pred_logits, p.features_out,
              ws_ptr<int>(p.ws, L.hdr) + H_STATUS};
   {

@@ -94,7 +94,12 @@ __host__ __device__ inline WsLayout ws_layout(int n_bs, int n_kv_heads, int num_
   // predictor front end: per (drafter-logit row, vocabulary chunk) a record of kPredRec
   // floats, per chunk the row sums of the fixed logit projection, per request the features
   L.pred_part = o;   o = ws_align(o + size_t(kPredPos) * n_bs * kPredMaxChunks * kPredRec * 4);
-  L.pred_rowsum = o; o = ws_align(o + size_t(kPredMaxChunks) * 32 * 4);
+  {
+    // partial row sums of the logit projection matrix: one vector of 32 per CTA of the stream grid
+    const int row_groups = (kPredPos * n_bs + 31) / 32;
+    const int slots = num_ctas > row_groups ? num_ctas : row_groups;
+    L.pred_rowsum = o; o = ws_align(o + size_t(slots > kPredMaxChunks ? slots : kPredMaxChunks) * 32 * 4);
+  }
   L.pred_feat = o;   o = ws_align(o + size_t(n_bs) * kPredFeatures * 4);
   // attention schedule: first linear key tile of every CTA's slice, [num_ctas + 1]
   L.slice_tab = o;   o = ws_align(o + (size_t(num_ctas) + 1) * 4);
