@@ -65,11 +65,6 @@ constexpr int kHidThreads = 256;                // threads of one hidden-project
 constexpr int kHidJobs = kWarps * 32 / kHidThreads;   // jobs side by side in a CTA that serves them
 constexpr int kHidSlices = 4;                   // 16 of the 64 outputs per job
 
-__device__ __forceinline__ float to_tf32(float x) {
-  uint32_t r;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-  return __uint_as_float(r);
-}
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -159,53 +154,54 @@ __device__ __forceinline__ void top16_offer_vec(float& tv, float& tau, float4 z,
   }
 }
 
-// running statistics of one logit row in one lane
+// Running statistics of one logit row in one lane.  `top` is the largest value of the row seen
+// so far by the whole warp (the head of the sorted list, the same in all lanes): it is the
+// reference of the exponentials, so the steady state needs no rescaling and the lanes' sums
+// are merged by plain addition.  A value above the reference is above the 16th as well, so
+// the reference only moves inside the (rare) list-update path.
 struct RowStat {
-  float m2, s, t, zsum;      // m2 = running max times log2(e)
+  float s, t, zsum;          // sum e, sum e z, sum z with e = exp(z - top)
+  float nref;                // -top log2(e); 0 while nothing finite has been seen
+  float top;
   float tv, tau;             // sorted top-16 (lane = rank) and the current 16th value
 };
 constexpr float kLog2e = 1.4426950408889634f;
-
-__device__ __forceinline__ void row_update(RowStat& r, float4 z, int c, int col_hi, int lane) {
-  const bool ragged = c + 3 >= col_hi;
-  if (ragged) {                                             // end of the vocabulary
-    if (c >= col_hi) z.x = -INFINITY;
-    if (c + 1 >= col_hi) z.y = -INFINITY;
-    if (c + 2 >= col_hi) z.z = -INFINITY;
-    z.w = -INFINITY;
-  }
-  const float zl = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
-  const float zl2 = zl * kLog2e;
-  if (zl2 > r.m2) {
-    const float f = ex2(r.m2 - zl2);                        // m2 = -inf gives 0
-    r.s *= f; r.t *= f; r.m2 = zl2;
-  }
-  const float zz[4] = {z.x, z.y, z.z, z.w};
-  if (!ragged) {
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      const float e = ex2(fmaf(zz[x], kLog2e, -r.m2));
-      r.s += e; r.t = fmaf(e, zz[x], r.t); r.zsum += zz[x];
-    }
-  } else {
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      if (zz[x] != -INFINITY) {
-        const float e = exp2f(fmaf(zz[x], kLog2e, -r.m2));
-        r.s += e; r.t = fmaf(e, zz[x], r.t); r.zsum += zz[x];
-      }
-    }
-  }
-  if (__any_sync(0xffffffffu, zl > r.tau)) {                // rare once the list has warmed up
-    top16_offer(r.tv, r.tau, z.x, lane);
-    top16_offer(r.tv, r.tau, z.y, lane);
-    top16_offer(r.tv, r.tau, z.z, lane);
-    top16_offer(r.tv, r.tau, z.w, lane);
+__device__ __forceinline__ void row_init(RowStat& r) {
+  r.s = r.t = r.zsum = r.nref = 0.f;
+  r.top = -INFINITY; r.tv = -INFINITY; r.tau = -INFINITY;
+}
+// the list-update path of one row: called by the whole warp when some lane may hold a value above the 16th
+__device__ __forceinline__ void row_event(RowStat& r, float4 z, float zl, int lane) {
+  top16_offer_vec(r.tv, r.tau, z, zl, lane);
+  const float nt = __shfl_sync(0xffffffffu, r.tv, 0);
+  if (nt > r.top) {                                         // a new maximum: move the reference
+    const float f = r.top == -INFINITY ? 0.f : ex2((r.top - nt) * kLog2e);
+    r.s *= f; r.t *= f;
+    r.top = nt;
+    r.nref = -(nt * kLog2e);
   }
 }
 
-// two rows at once: the same arithmetic as row_update, written so that the two rows'
-// chains are independent instructions of one basic block
+// one row, the careful path for the end of the vocabulary: values at or beyond col_hi do not count
+__device__ __forceinline__ void row_update(RowStat& r, float4 z, int c, int col_hi, int lane) {
+  if (c >= col_hi) z.x = -INFINITY;
+  if (c + 1 >= col_hi) z.y = -INFINITY;
+  if (c + 2 >= col_hi) z.z = -INFINITY;
+  if (c + 3 >= col_hi) z.w = -INFINITY;
+  const float zl = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
+  if (__any_sync(0xffffffffu, zl > r.tau)) row_event(r, z, zl, lane);
+  const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {
+    if (zz[x] != -INFINITY) {
+      const float e = ex2(fmaf(zz[x], kLog2e, r.nref));
+      r.s += e; r.t = fmaf(e, zz[x], r.t); r.zsum += zz[x];
+    }
+  }
+}
+
+// two rows at once, written so that the two rows' chains are independent instructions of one
+// basic block
 __device__ __forceinline__ void row_update2(RowStat& a, RowStat& b, float4 za, float4 zb, int c, int col_hi,
                                             int lane) {
   if (c - 4 * lane + kSub > col_hi) {                       // ragged end (warp-uniform test): the careful path
@@ -215,21 +211,18 @@ __device__ __forceinline__ void row_update2(RowStat& a, RowStat& b, float4 za, f
   }
   const float la = fmaxf(fmaxf(za.x, za.y), fmaxf(za.z, za.w));
   const float lb = fmaxf(fmaxf(zb.x, zb.y), fmaxf(zb.z, zb.w));
-  const float na = fmaxf(a.m2, la * kLog2e), nb = fmaxf(b.m2, lb * kLog2e);
-  const float fa = ex2(a.m2 - na), fb = ex2(b.m2 - nb);     // 1 when the maximum stands; m2 = -inf gives 0
-  a.s *= fa; a.t *= fa; a.m2 = na;
-  b.s *= fb; b.t *= fb; b.m2 = nb;
+  if (__any_sync(0xffffffffu, la > a.tau || lb > b.tau)) {  // rare once the lists have warmed up
+    if (__any_sync(0xffffffffu, la > a.tau)) row_event(a, za, la, lane);
+    if (__any_sync(0xffffffffu, lb > b.tau)) row_event(b, zb, lb, lane);
+  }
+  const float na = a.nref, nb = b.nref;
   const float xa[4] = {za.x, za.y, za.z, za.w}, xb[4] = {zb.x, zb.y, zb.z, zb.w};
 #pragma unroll
   for (int x = 0; x < 4; ++x) {
-    const float ea = ex2(fmaf(xa[x], kLog2e, -na)), eb = ex2(fmaf(xb[x], kLog2e, -nb));
+    const float ea = ex2(fmaf(xa[x], kLog2e, na)), eb = ex2(fmaf(xb[x], kLog2e, nb));
     a.s += ea; b.s += eb;
     a.t = fmaf(ea, xa[x], a.t); b.t = fmaf(eb, xb[x], b.t);
     a.zsum += xa[x]; b.zsum += xb[x];
-  }
-  if (__any_sync(0xffffffffu, la > a.tau || lb > b.tau)) {  // rare once the lists have warmed up
-    top16_offer_vec(a.tv, a.tau, za, la, lane);
-    top16_offer_vec(b.tv, b.tau, zb, lb, lane);
   }
 }
 
@@ -415,10 +408,7 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
   }
 
   RowStat rs[2];
-#pragma unroll
-  for (int x = 0; x < 2; ++x) {
-    rs[x].m2 = -INFINITY; rs[x].s = 0.f; rs[x].t = 0.f; rs[x].zsum = 0.f; rs[x].tv = -INFINITY; rs[x].tau = -INFINITY;
-  }
+  row_init(rs[0]); row_init(rs[1]);
   float p_rowsum = 0.f;
   float d[2][4][4];
 #pragma unroll
@@ -468,10 +458,12 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
         const float2 zlo = *reinterpret_cast<const float2*>(zst + zo[2 * h]);
         const float2 zhi = *reinterpret_cast<const float2*>(zst + zo[2 * h + 1]);
         uint32_t af[4];
-        af[0] = __float_as_uint(to_tf32(zlo.x - piv[2 * h]));
-        af[1] = __float_as_uint(to_tf32(zhi.x - piv[2 * h + 1]));
-        af[2] = __float_as_uint(to_tf32(zlo.y - piv[2 * h]));
-        af[3] = __float_as_uint(to_tf32(zhi.y - piv[2 * h + 1]));
+        // z - pivot, rounded to tf32 the way cvt.rna does (add half a tf32 ulp to the bit pattern;
+        // the tensor core ignores the low 13 bits), on the integer pipe instead of the conversion unit
+        af[0] = __float_as_uint(zlo.x - piv[2 * h]) + 0x1000u;
+        af[1] = __float_as_uint(zhi.x - piv[2 * h + 1]) + 0x1000u;
+        af[2] = __float_as_uint(zlo.y - piv[2 * h]) + 0x1000u;
+        af[3] = __float_as_uint(zhi.y - piv[2 * h + 1]) + 0x1000u;
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) mma_tf32(d[h][nt], af, bw[nt] << 16, bw[nt] & 0xffff0000u);
       }
@@ -498,26 +490,20 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
     return;
   }
 
-  // ---- row statistics: merge the 32 lanes, write the records
+  // ---- row statistics: merge the 32 lanes (one reference per row: plain sums), write the records
 #pragma unroll
   for (int x = 0; x < 2; ++x) {
-    float m2 = rs[x].m2, s_sum = rs[x].s, t_sum = rs[x].t, z_sum = rs[x].zsum;
+    float s_sum = rs[x].s, t_sum = rs[x].t, z_sum = rs[x].zsum;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-      const float mo = __shfl_xor_sync(0xffffffffu, m2, o);
-      const float s2 = __shfl_xor_sync(0xffffffffu, s_sum, o);
-      const float t2 = __shfl_xor_sync(0xffffffffu, t_sum, o);
+      s_sum += __shfl_xor_sync(0xffffffffu, s_sum, o);
+      t_sum += __shfl_xor_sync(0xffffffffu, t_sum, o);
       z_sum += __shfl_xor_sync(0xffffffffu, z_sum, o);
-      const float mm = fmaxf(m2, mo);
-      const float r1 = m2 == -INFINITY ? 0.f : exp2f(m2 - mm), r2 = mo == -INFINITY ? 0.f : exp2f(mo - mm);
-      s_sum = s_sum * r1 + s2 * r2;
-      t_sum = t_sum * r1 + t2 * r2;
-      m2 = mm;
     }
     if (live[x]) {
       float* rec = a.part + ((size_t)my_row[x] * a.chunks + chunk) * kPredRec;
       if (lane < 16) rec[lane] = rs[x].tv;
-      if (lane == 0) { rec[16] = m2 / kLog2e; rec[17] = s_sum; rec[18] = t_sum; rec[19] = z_sum; }
+      if (lane == 0) { rec[16] = rs[x].top; rec[17] = s_sum; rec[18] = t_sum; rec[19] = z_sum; }
     }
   }
   // ---- projection: sum the 16 warps' k slices through shared memory (the ring is idle now)
