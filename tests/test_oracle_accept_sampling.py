@@ -65,6 +65,27 @@ def test_acceptance_threshold_and_all_pass():
     assert r["accept_len"][0] == 1 and r["out_tokens"][0, 0] == 4
 
 
+def test_all_pass_draws_from_the_last_rows_unmodified_distribution():
+    """When every candidate passes, the successor comes from the last selected row's P as it
+    stands ("Prefix verifier" paragraph): no token is removed, the last candidate itself can be
+    drawn again.  The last row's P is fixed by hand (logits = log of 0.1, 0.2, 0.3, 0.4), so the
+    expected token for each uniform follows from the cumulative sums 0.1, 0.3, 0.6, 1.0."""
+    probs = np.array([0.1, 0.2, 0.3, 0.4])
+    rows = np.zeros((3, 4), dtype=np.float32)                 # rows 0 and 1: uniform P = 1/4 each
+    rows[2] = np.log(probs).astype(np.float32)
+    toks = [0, 2, 3]                                          # anchor, candidates 2 and 3
+    for u, want in ((0.05, 0), (0.15, 1), (0.29, 1), (0.31, 2), (0.59, 2), (0.61, 3), (0.95, 3)):
+        r = _single(rows, toks, [0.2, 0.2], u)                # 0.2 < 1/4: both candidates pass
+        assert r["accept_len"][0] == 2 and r["out_len"][0] == 3
+        assert r["next_anchor"][0] == want, (u, r["next_anchor"][0])
+        assert list(r["out_tokens"][0, :3]) == [2, 3, want]
+    # the same uniforms after a rejection of candidate 3 at row 1 draw from row 1's P without token 3:
+    # uniform over {0, 1, 2}, thirds
+    for u, want in ((0.1, 0), (0.4, 1), (0.9, 2)):
+        r = _single(rows, toks, [0.2, 0.3], u)                # 0.3 > 1/4: the second candidate is rejected
+        assert r["accept_len"][0] == 1 and r["next_anchor"][0] == want, (u, r["next_anchor"][0])
+
+
 def test_low_temperature_reduces_to_greedy():
     """As the temperature goes to 0 the policy puts all mass on the arg-max: sampling
     verification must then return exactly the greedy result, whatever the uniforms."""
