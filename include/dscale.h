@@ -239,8 +239,10 @@ int dscale_accept(void* ws, int n_bs, const float* logits, int64_t ld, int vocab
  * memory into `staging`, the three stages are enqueued (allocation, attention
  * for each of n_layers layers, acceptance), and the outputs are copied back to
  * host memory, all asynchronously on `stream`; the results are valid after the
- * caller synchronises the stream.  Host buffers should be page-locked for the
- * copies to be asynchronous.
+ * caller synchronises the stream.  Host buffers should be page-locked: the
+ * staged inputs are then fetched, and the results written back, by one small
+ * kernel each over the buffers' device mapping (2 launches more per step);
+ * pageable buffers are served by ordinary copies, which are then not asynchronous.
  *
  *   h_*          HOST pointers, same shapes as in the per-stage calls
  *   staging      DEVICE scratch of at least dscale_step_staging_bytes(n_bs, max_pages)

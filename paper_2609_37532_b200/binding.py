@@ -205,11 +205,11 @@ class HostStep:
     stream and returns without synchronising."""
 
     def __init__(self, ws: VerifyWorkspace, max_pages: int, num_pages: int, layers, logits,
-                 vocab: int, sm_scale: float):
+                 vocab: int, sm_scale: float, pinned: bool = True):
         n_bs = ws.n_bs
         self.ws, self.max_pages, self.num_pages = ws, max_pages, num_pages
         self.vocab, self.sm_scale, self.logits = vocab, float(sm_scale), logits
-        pin = dict(pin_memory=True)
+        pin = dict(pin_memory=pinned)       # pageable buffers take the library's copy path
         self.h_n_live = torch.zeros(1, dtype=torch.int32, **pin)
         self.h_scores = torch.zeros((n_bs, 15), dtype=torch.float32, **pin)
         self.h_draft = torch.zeros((n_bs, 16), dtype=torch.int32, **pin)

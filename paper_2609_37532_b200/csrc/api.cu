@@ -230,6 +230,39 @@ StagingLayout staging_layout(int n_bs, int max_pages) {
   S.total = o;
   return S;
 }
+
+// Stage-in / stage-out for the host-buffer step.  Page-locked host memory is mapped into the
+// device's address space, so one small kernel can fetch all five staged inputs of a step over
+// the bus at once (65 KB at n_bs = 32), and another can write the four results back, instead
+// of nine copy operations that run one after another with a fixed cost each (about 10 us per
+// copy on this class of machine).  Memory that is not mapped (pageable buffers) takes the
+// copy path.
+constexpr int kStageRegions = 5;
+struct StageCopy {
+  const uint32_t* src[kStageRegions];
+  uint32_t* dst[kStageRegions];
+  int words[kStageRegions];
+  int n;
+};
+__global__ void stage_copy_kernel(StageCopy c) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x, nt = gridDim.x * blockDim.x;
+  for (int r = 0; r < c.n; ++r)
+    for (int i = t; i < c.words[r]; i += nt) c.dst[r][i] = c.src[r][i];
+}
+// the device's view of a page-locked host buffer, or nullptr if the device cannot address it
+const void* mapped(const void* host) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, host) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  if (at.type != cudaMemoryTypeHost) return nullptr;
+  return at.devicePointer;
+}
+bool launch_stage_copy(const StageCopy& c, cudaStream_t st) {
+  int total = 0;
+  for (int r = 0; r < c.n; ++r) total += c.words[r];
+  const int blocks = total / (256 * 8) < 1 ? 1 : (total / (256 * 8) > 32 ? 32 : total / (256 * 8));
+  stage_copy_kernel<<<blocks, 256, 0, st>>>(c);
+  return cudaGetLastError() == cudaSuccess;
+}
 }  // namespace
 
 size_t dscale_step_staging_bytes(int n_bs, int max_pages) {
@@ -258,11 +291,26 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
   auto d2h = [&](void* dst, size_t off, size_t bytes) {
     return cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   };
-  if (!h2d(S.n_live, h_n_live, 4) || !h2d(S.scores, h_scores, size_t(n_bs) * 15 * 4) ||
-      !h2d(S.draft, h_draft_tokens, size_t(n_bs) * 16 * 4) ||
-      !h2d(S.ctx_len, h_ctx_len, size_t(n_bs) * 4) ||
-      !h2d(S.block_table, h_block_table, size_t(n_bs) * max_pages * 4))
-    return DSCALE_ERR_CUDA;
+  {
+    const void* hp[kStageRegions] = {h_n_live, h_scores, h_draft_tokens, h_ctx_len, h_block_table};
+    const size_t off[kStageRegions] = {S.n_live, S.scores, S.draft, S.ctx_len, S.block_table};
+    const int words[kStageRegions] = {1, n_bs * 15, n_bs * 16, n_bs, n_bs * max_pages};
+    StageCopy c;
+    c.n = kStageRegions;
+    bool all_mapped = true;
+    for (int r = 0; r < kStageRegions; ++r) {
+      c.src[r] = static_cast<const uint32_t*>(mapped(hp[r]));
+      c.dst[r] = reinterpret_cast<uint32_t*>(d + off[r]);
+      c.words[r] = words[r];
+      all_mapped = all_mapped && c.src[r] != nullptr;
+    }
+    if (all_mapped) {
+      if (!launch_stage_copy(c, st)) return DSCALE_ERR_CUDA;
+    } else {
+      for (int r = 0; r < kStageRegions; ++r)
+        if (!h2d(off[r], hp[r], size_t(words[r]) * 4)) return DSCALE_ERR_CUDA;
+    }
+  }
   const int32_t* d_bt = reinterpret_cast<const int32_t*>(d + S.block_table);
   int rc = dscale_alloc_verify(ws, n_bs, reinterpret_cast<const int32_t*>(d + S.n_live),
                                reinterpret_cast<const float*>(d + S.scores), 0,
@@ -281,11 +329,26 @@ int dscale_verify_step_host(void* ws, int n_bs, const int32_t* h_n_live, const f
                      reinterpret_cast<int32_t*>(d + S.out_tokens),
                      reinterpret_cast<int32_t*>(d + S.out_len), nullptr, stream);
   if (rc != DSCALE_OK) return rc;
-  if (!d2h(h_accept_len, S.accept_len, size_t(n_bs) * 4) ||
-      !d2h(h_next_anchor, S.next_anchor, size_t(n_bs) * 4) ||
-      !d2h(h_out_tokens, S.out_tokens, size_t(n_bs) * 16 * 4) ||
-      !d2h(h_out_len, S.out_len, size_t(n_bs) * 4))
-    return DSCALE_ERR_CUDA;
+  {
+    void* hp[4] = {h_accept_len, h_next_anchor, h_out_tokens, h_out_len};
+    const size_t off[4] = {S.accept_len, S.next_anchor, S.out_tokens, S.out_len};
+    const int words[4] = {n_bs, n_bs, n_bs * 16, n_bs};
+    StageCopy c;
+    c.n = 4;
+    bool all_mapped = true;
+    for (int r = 0; r < 4; ++r) {
+      c.dst[r] = static_cast<uint32_t*>(const_cast<void*>(mapped(hp[r])));
+      c.src[r] = reinterpret_cast<const uint32_t*>(d + off[r]);
+      c.words[r] = words[r];
+      all_mapped = all_mapped && c.dst[r] != nullptr;
+    }
+    if (all_mapped) {
+      if (!launch_stage_copy(c, st)) return DSCALE_ERR_CUDA;
+    } else {
+      for (int r = 0; r < 4; ++r)
+        if (!d2h(hp[r], off[r], size_t(words[r]) * 4)) return DSCALE_ERR_CUDA;
+    }
+  }
   return DSCALE_OK;
 }
 

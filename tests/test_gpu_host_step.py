@@ -10,8 +10,10 @@ from gpu_case import SCALE, attn_close, oracle_accept, oracle_alloc, oracle_attn
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("n_layers", [1, 3])
-def test_host_step_matches_oracle(n_layers):
+@pytest.mark.parametrize("n_layers,pinned", [(1, True), (3, True), (2, False)])
+def test_host_step_matches_oracle(n_layers, pinned):
+    """pinned: the staged inputs and the results travel through the buffers' device mapping (one
+    small kernel each way); pageable: through ordinary copies."""
     import paper_2609_37532_b200 as P
     cfg = small_variant(CONFIGS["tiny"], vocab=5000, n=6, seed=31, ctx_lo=10, ctx_hi=700)
     req = make_requests(cfg, n_bs=8)
@@ -26,7 +28,8 @@ def test_host_step_matches_oracle(n_layers):
         layers.append((qp.cuda().contiguous(), kc.cuda(), vc.cuda(),
                        torch.full(qp.shape, float("nan"), dtype=torch.bfloat16, device="cuda")))
     lp = rows_to_packed(make_logits_unpacked(req), alloc["k"], alloc["offset"], n, 8 * n_bs)
-    hs = P.HostStep(ws, req["max_pages"], req["num_pages"], layers, lp.cuda().contiguous(), cfg.vocab, SCALE)
+    hs = P.HostStep(ws, req["max_pages"], req["num_pages"], layers, lp.cuda().contiguous(), cfg.vocab, SCALE,
+                    pinned=pinned)
     hs.h_n_live[0] = n
     hs.h_scores.copy_(torch.as_tensor(req["scores"]))
     hs.h_draft.copy_(torch.as_tensor(req["draft_tokens"]))
