@@ -79,6 +79,7 @@ def _case(P, cfg, n_bs, hidden_dim, gen_device="cpu"):
     (20, 17, 50000, 512),     # several row groups and chunks, a ragged last chunk
     (64, 64, 4096, 128),      # largest capacity
     (2, 1, 16, 8),            # smallest legal shapes
+    (32, 5, 20480, 256),      # few live requests in a large capacity: most row groups dead, the live ones share the row sums
 ])
 def test_predictor_small_shapes(n_bs, n, vocab, hidden_dim):
     import paper_2609_37532_b200 as P
