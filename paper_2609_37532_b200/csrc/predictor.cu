@@ -139,21 +139,6 @@ __device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// offer the four values of every lane: the lane maxima first (one round), and the other three
-// only if one of them still beats the 16th afterwards (an event usually brings a single value)
-__device__ __forceinline__ void top16_offer_vec(float& tv, float& tau, float4 z, float zmax, int lane) {
-  if (!__any_sync(0xffffffffu, zmax > tau)) return;
-  top16_offer(tv, tau, zmax, lane);
-  // the remaining three: the first component equal to the maximum is the one already offered
-  const bool mx = z.x == zmax, my = !mx && z.y == zmax, mz = !mx && !my && z.z == zmax;
-  const float rx = mx ? -INFINITY : z.x, ry = my ? -INFINITY : z.y, rz = mz ? -INFINITY : z.z;
-  const float rw = (mx || my || mz) ? z.w : -INFINITY;
-  if (__any_sync(0xffffffffu, fmaxf(fmaxf(rx, ry), fmaxf(rz, rw)) > tau)) {
-    top16_offer(tv, tau, rx, lane); top16_offer(tv, tau, ry, lane);
-    top16_offer(tv, tau, rz, lane); top16_offer(tv, tau, rw, lane);
-  }
-}
-
 // Running statistics of one logit row in one lane.  `top` is the largest value of the row seen
 // so far by the whole warp (the head of the sorted list, the same in all lanes): it is the
 // reference of the exponentials, so the steady state needs no rescaling and the lanes' sums
@@ -170,15 +155,50 @@ __device__ __forceinline__ void row_init(RowStat& r) {
   r.s = r.t = r.zsum = r.nref = 0.f;
   r.top = -INFINITY; r.tv = -INFINITY; r.tau = -INFINITY;
 }
-// the list-update path of one row: called by the whole warp when some lane may hold a value above the 16th
-__device__ __forceinline__ void row_event(RowStat& r, float4 z, float zl, int lane) {
-  top16_offer_vec(r.tv, r.tau, z, zl, lane);
-  const float nt = __shfl_sync(0xffffffffu, r.tv, 0);
-  if (nt > r.top) {                                         // a new maximum: move the reference
-    const float f = r.top == -INFINITY ? 0.f : ex2((r.top - nt) * kLog2e);
+// The list-update path of one row: called by the whole warp with the ballot of the lanes whose
+// maximum beats the 16th.  What a warp pays here is latency, a chain of warp collectives, so the
+// chain is kept short: the candidates are inserted one after another without looking at the new
+// 16th in between (a value that is too small changes no lane), whether some lane holds a SECOND
+// value above the 16th is decided up front against the old threshold (rare; then the other three
+// values of every lane are offered as well), the new 16th is fetched once at the end, and the
+// row maximum follows from the candidates themselves.
+__device__ __forceinline__ void row_event(RowStat& r, float4 z, float zl, unsigned cand, int lane) {
+  const float m01 = fmaxf(z.x, z.y), n01 = fminf(z.x, z.y), m23 = fmaxf(z.z, z.w), n23 = fminf(z.z, z.w);
+  const float second = fmaxf(fminf(m01, m23), m01 >= m23 ? n01 : n23);   // second largest of the four
+  const bool more = __any_sync(0xffffffffu, second > r.tau);
+  float vmax = -INFINITY;                                   // warp-uniform: the largest candidate
+  while (cand) {
+    const int src = __ffs(cand) - 1;
+    cand &= cand - 1;
+    const float v = __shfl_sync(0xffffffffu, zl, src);
+    top16_insert(r.tv, v, lane);
+    vmax = fmaxf(vmax, v);
+  }
+  r.tau = __shfl_sync(0xffffffffu, r.tv, 15);
+  if (more) {
+    // the first component equal to the maximum is the one already offered; the others are offered
+    // component by component against the 16th as it stands, which is fetched once per component
+    const bool mx = z.x == zl, my = !mx && z.y == zl, mz = !mx && !my && z.z == zl;
+    const float rest[4] = {mx ? -INFINITY : z.x, my ? -INFINITY : z.y, mz ? -INFINITY : z.z,
+                           (mx || my || mz) ? z.w : -INFINITY};
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      unsigned m = __ballot_sync(0xffffffffu, rest[x] > r.tau);
+      if (m) {
+        while (m) {
+          const int src = __ffs(m) - 1;
+          m &= m - 1;
+          top16_insert(r.tv, __shfl_sync(0xffffffffu, rest[x], src), lane);
+        }
+        r.tau = __shfl_sync(0xffffffffu, r.tv, 15);
+      }
+    }
+  }
+  if (vmax > r.top) {                                       // a new maximum: move the reference
+    const float f = r.top == -INFINITY ? 0.f : ex2((r.top - vmax) * kLog2e);
     r.s *= f; r.t *= f;
-    r.top = nt;
-    r.nref = -(nt * kLog2e);
+    r.top = vmax;
+    r.nref = -(vmax * kLog2e);
   }
 }
 
@@ -189,7 +209,8 @@ __device__ __forceinline__ void row_update(RowStat& r, float4 z, int c, int col_
   if (c + 2 >= col_hi) z.z = -INFINITY;
   if (c + 3 >= col_hi) z.w = -INFINITY;
   const float zl = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
-  if (__any_sync(0xffffffffu, zl > r.tau)) row_event(r, z, zl, lane);
+  const unsigned cand = __ballot_sync(0xffffffffu, zl > r.tau);
+  if (cand) row_event(r, z, zl, cand, lane);
   const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
   for (int x = 0; x < 4; ++x) {
@@ -212,8 +233,9 @@ __device__ __forceinline__ void row_update2(RowStat& a, RowStat& b, float4 za, f
   const float la = fmaxf(fmaxf(za.x, za.y), fmaxf(za.z, za.w));
   const float lb = fmaxf(fmaxf(zb.x, zb.y), fmaxf(zb.z, zb.w));
   if (__any_sync(0xffffffffu, la > a.tau || lb > b.tau)) {  // rare once the lists have warmed up
-    if (__any_sync(0xffffffffu, la > a.tau)) row_event(a, za, la, lane);
-    if (__any_sync(0xffffffffu, lb > b.tau)) row_event(b, zb, lb, lane);
+    const unsigned ca = __ballot_sync(0xffffffffu, la > a.tau), cb = __ballot_sync(0xffffffffu, lb > b.tau);
+    if (ca) row_event(a, za, la, ca, lane);
+    if (cb) row_event(b, zb, lb, cb, lane);
   }
   const float na = a.nref, nb = b.nref;
   const float xa[4] = {za.x, za.y, za.z, za.w}, xb[4] = {zb.x, zb.y, zb.z, zb.w};
