@@ -62,6 +62,20 @@ __global__ void __launch_bounds__(kAccThreads, 2) accept_kernel(AcceptArgs a, Ws
   const int tid = threadIdx.x, lane = tid & 31;
   unsigned long long* row_key = ws_ptr<unsigned long long>(a.ws, L.amax_val);   // [8 n_bs], 0 = untouched
   __shared__ int sLast;
+  // The acceptance loop at the end is a chain of dependent reads: it runs on shared-memory copies
+  // of the per-row results and of the packed tokens, lengths and offsets.  The copies of the
+  // allocation's outputs are fetched now, by every CTA (2 KB, from L2), so that the one CTA that
+  // ends up last does not start a round of loads when everybody else has already left.
+  __shared__ int s_top1[kHalfW * kMaxNbs];
+  __shared__ int s_tok[kHalfW * kMaxNbs];
+  __shared__ int s_k[kMaxNbs], s_off[kMaxNbs];
+  {
+    const int* wtok = ws_ptr<int>(a.ws, L.tokens);
+    const int* wk = ws_ptr<int>(a.ws, L.k);
+    const int* woff = ws_ptr<int>(a.ws, L.offset);
+    for (int r = tid; r < kHalfW * a.n_bs; r += kAccThreads) s_tok[r] = wtok[r];
+    for (int r = tid; r < a.n_bs; r += kAccThreads) { s_k[r] = wk[r]; s_off[r] = woff[r]; }
+  }
 
   // this warp's span of the ragged vector sequence
   const long long nv = (a.vocab + 3) >> 2;                      // vectors per row
@@ -117,12 +131,7 @@ __global__ void __launch_bounds__(kAccThreads, 2) accept_kernel(AcceptArgs a, Ws
   if (tid == 0) hdr[H_ACCEPT_TICKET] = 0;           // ready for the next replay
   const int n_bs = a.n_bs;
   const int m_bs = kHalfW * n_bs;
-  // The acceptance loop is a chain of dependent reads: run it on shared-memory copies
-  // of the per-row results and the packed tokens, not on global memory.
-  __shared__ int s_top1[kHalfW * kMaxNbs];
-  __shared__ int s_tok[kHalfW * kMaxNbs];
   int* top1 = ws_ptr<int>(a.ws, L.top1);
-  const int* wtok = ws_ptr<int>(a.ws, L.tokens);
   for (int r = tid; r < m_bs; r += kAccThreads) {
     int best = 0;
     if (r < m_live) {
@@ -132,16 +141,13 @@ __global__ void __launch_bounds__(kAccThreads, 2) accept_kernel(AcceptArgs a, Ws
     }
     top1[r] = best;
     s_top1[r] = best;
-    s_tok[r] = wtok[r];
   }
   __syncthreads();
   const int N = hdr[H_N_LIVE];
-  const int* wk = ws_ptr<int>(a.ws, L.k);
-  const int* woff = ws_ptr<int>(a.ws, L.offset);
   for (int i = tid; i < n_bs; i += kAccThreads) {
     int* ot = a.out_tokens + i * kW;
     if (i < N) {
-      const int ki = wk[i], oi = woff[i];
+      const int ki = s_k[i], oi = s_off[i];
       int acc = 0;
       while (acc < ki - 1 && s_top1[oi + acc] == s_tok[oi + acc + 1]) ++acc;
       const int nxt = s_top1[oi + acc];
