@@ -155,6 +155,32 @@ __device__ __forceinline__ void row_init(RowStat& r) {
   r.s = r.t = r.zsum = r.nref = 0.f;
   r.top = -INFINITY; r.tv = -INFINITY; r.tau = -INFINITY;
 }
+// The rare part of a list update: some lane holds a second value above the 16th.  The first
+// component equal to the lane's maximum is the one already offered; the others are offered
+// component by component against the 16th as it stands, which is fetched once per component.
+// Kept out of line: it runs a few times per row and chunk, and inlined (twice, unrolled four times)
+// it made the hot loop larger and the whole kernel 1 us slower.  Returns (list entry
+// of this lane, new 16th).
+__device__ __noinline__ float2 offer_rest(float tv, float tau, float4 z, float zl, int lane) {
+  const bool mx = z.x == zl, my = !mx && z.y == zl, mz = !mx && !my && z.z == zl;
+  const float rest[4] = {mx ? -INFINITY : z.x, my ? -INFINITY : z.y, mz ? -INFINITY : z.z,
+                         (mx || my || mz) ? z.w : -INFINITY};
+#pragma unroll 1
+  for (int x = 0; x < 4; ++x) {
+    const float rv = x == 0 ? rest[0] : (x == 1 ? rest[1] : (x == 2 ? rest[2] : rest[3]));
+    unsigned m = __ballot_sync(0xffffffffu, rv > tau);
+    if (m) {
+      while (m) {
+        const int src = __ffs(m) - 1;
+        m &= m - 1;
+        top16_insert(tv, __shfl_sync(0xffffffffu, rv, src), lane);
+      }
+      tau = __shfl_sync(0xffffffffu, tv, 15);
+    }
+  }
+  return make_float2(tv, tau);
+}
+
 // The list-update path of one row: called by the whole warp with the ballot of the lanes whose
 // maximum beats the 16th.  What a warp pays here is latency, a chain of warp collectives, so the
 // chain is kept short: the candidates are inserted one after another without looking at the new
@@ -176,23 +202,8 @@ __device__ __forceinline__ void row_event(RowStat& r, float4 z, float zl, unsign
   }
   r.tau = __shfl_sync(0xffffffffu, r.tv, 15);
   if (more) {
-    // the first component equal to the maximum is the one already offered; the others are offered
-    // component by component against the 16th as it stands, which is fetched once per component
-    const bool mx = z.x == zl, my = !mx && z.y == zl, mz = !mx && !my && z.z == zl;
-    const float rest[4] = {mx ? -INFINITY : z.x, my ? -INFINITY : z.y, mz ? -INFINITY : z.z,
-                           (mx || my || mz) ? z.w : -INFINITY};
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      unsigned m = __ballot_sync(0xffffffffu, rest[x] > r.tau);
-      if (m) {
-        while (m) {
-          const int src = __ffs(m) - 1;
-          m &= m - 1;
-          top16_insert(r.tv, __shfl_sync(0xffffffffu, rest[x], src), lane);
-        }
-        r.tau = __shfl_sync(0xffffffffu, r.tv, 15);
-      }
-    }
+    const float2 lt = offer_rest(r.tv, r.tau, z, zl, lane);
+    r.tv = lt.x; r.tau = lt.y;
   }
   if (vmax > r.top) {                                       // a new maximum: move the reference
     const float f = r.top == -INFINITY ? 0.f : ex2((r.top - vmax) * kLog2e);
