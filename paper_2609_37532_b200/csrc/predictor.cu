@@ -3,22 +3,22 @@
 // paragraph, Eq. 4 and Eq. 5).  Two launches (the tail is scheduled while the stream runs):
 //
 //  pred_stream_kernel    the only pass over the drafter logits (15 N rows x V fp32,
-//                        292 MB at N = 32: an HBM stream).  A CTA of 16 warps owns
-//                        16 rows x one vocabulary chunk; warp w streams row w with
-//                        coalesced 128-bit loads and keeps, per row, the running
-//                        (max, sum e^{z-max}, sum e^{z-max} z, sum z) and the 16
-//                        largest values (sorted in lanes 0-15; a new value enters
-//                        only if it beats the 16th, found by a warp ballot, so the
-//                        steady state costs one compare per element).  The fixed
-//                        32 x V logit projection is a dense contraction with K = V:
-//                        every 128-column sub-tile is also stored to shared memory
-//                        (minus a per-row pivot, rounded to tf32) next to the
-//                        matching 32 x 128 tile of the projection matrix, and the
-//                        16 warps each issue one k = 8 step of m16n8k8 tf32 MMAs
-//                        over it.  Warp-level MMAs on purpose: 4.7 GFLOP ride
-//                        along with a 292 MB stream, there is no tensor-core
-//                        time to win, and the rows are already in registers.
-//                        One record per (row, chunk) goes to the workspace.
+//                        292 MB at N = 32: an HBM stream).  A CTA of 16 compute warps
+//                        and a copy warp owns 32 rows x one vocabulary chunk; the copy
+//                        warp fills a shared-memory ring with TMA boxes, warp w streams
+//                        rows w and w + 16 with 128-bit shared loads and keeps, per row,
+//                        the running (sum e^{z-top}, sum e^{z-top} z, sum z) and the 16
+//                        largest values (sorted in lanes 0-15; a new value enters only
+//                        if it beats the 16th, found by a warp vote, so the steady state
+//                        costs one compare per four elements; `top`, the reference of
+//                        the exponentials, is the head of that list).  The fixed 32 x V
+//                        logit projection is a dense contraction with K = V: next to
+//                        every 128-column sub-tile of logits the ring holds the matching
+//                        32 x 128 tile of the projection matrix, and the 16 warps each
+//                        issue one k = 8 step of m16n8k8 tf32 MMAs over it (operands
+//                        z - pivot, rounded to tf32).  Warp-level MMAs on purpose: 4.7
+//                        GFLOP ride along with a 292 MB stream, there is no tensor-core
+//                        time to win.  One record per (row, chunk) goes to the workspace.
 //                        The CTAs of the grid behind the (row group, chunk) CTAs compute
 //                        the 64 x H hidden-state projection of all rows (bf16 MMAs) on
 //                        the SMs the stream leaves free.
