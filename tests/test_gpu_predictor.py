@@ -136,3 +136,36 @@ def test_predictor_rejects_bad_shapes():
     nl = torch.ones(1, dtype=torch.int32, device="cuda")
     with pytest.raises(RuntimeError):
         P.predict_scores(ws, nl, z, 1002, h, ph, pl, w1, b1, w2, b2, out)
+
+
+def test_predictor_w1_not_16_byte_aligned_and_no_live_requests():
+    """Two corners of the tail kernel: W1 at an address that is not a multiple of 16 bytes (no bulk
+    copy into shared memory: the rows are read from global memory, same arithmetic, same result),
+    and a call with no live request (all outputs zero, nothing read)."""
+    import paper_2609_37532_b200 as P
+    cfg = small_variant(CONFIGS["tiny"], vocab=4096, n=3, seed=79)
+    req = make_requests(cfg, n_bs=4)
+    d = {k: (v.cuda().contiguous() if torch.is_tensor(v) else v) for k, v in make_predictor_inputs(req, 64).items()}
+    ws = P.VerifyWorkspace(4, cfg.n_q_heads, cfg.n_kv_heads)
+    st = StagedRequests(req)
+
+    def run(w1, n_live):
+        pred = torch.full((4, 15), 7.0, dtype=torch.float32, device="cuda")
+        feat = torch.full((4, 1735), 7.0, dtype=torch.float32, device="cuda")
+        P.predict_scores(ws, n_live, d["draft_logits"], 4096, d["draft_hidden"], d["p_hidden"], d["p_logit"],
+                         w1, d["b1"], d["w2"], d["b2"], pred, feat)
+        torch.cuda.synchronize()
+        assert ws.status() == 0
+        return pred.cpu().numpy(), feat.cpu().numpy()
+
+    base_pred, base_feat = run(d["w1"], st.n_live)
+    shifted = torch.zeros(64 * 1735 + 1, dtype=torch.float32, device="cuda")
+    w1m = shifted[1:].view(64, 1735)
+    w1m.copy_(d["w1"])
+    assert w1m.data_ptr() % 16 == 4
+    pred, feat = run(w1m, st.n_live)
+    np.testing.assert_array_equal(pred, base_pred)
+    np.testing.assert_array_equal(feat, base_feat)
+    none = torch.zeros(1, dtype=torch.int32, device="cuda")
+    pred, feat = run(d["w1"], none)
+    assert (pred == 0).all() and (feat == 0).all()
