@@ -35,6 +35,10 @@
 
 namespace dscale {
 
+#ifdef DSCALE_WAIT_TEST
+__device__ int g_pred_drop_cta = -1, g_pred_drop_sub = -1;
+#endif
+
 namespace {
 
 constexpr int kWarps = 16;                      // warps per CTA = k steps of 8 per sub-tile
@@ -419,8 +423,15 @@ pred_stream_kernel(StreamArgs a, const __grid_constant__ CUtensorMap tm_z, const
       const int c = col_lo + v * kSub;
       if (lane == 0) mbar_expect_tx(full(st), kZStage + (p_vec ? kPStage : 0));
       __syncwarp();
-      if (lane < 4) tma_box_2d(sbase + st * kZStage + lane * (kRowsPerCta * 128), &tm_z, full(st), c + 32 * lane, row0);
-      else if (lane < 6 && p_vec)
+#ifdef DSCALE_WAIT_TEST
+      // wait-limit test build only: the logit boxes of one sub-tile of one CTA are left out (the
+      // barrier stays armed), so that every wait behind it runs into its limit
+      const bool drop = (int)blockIdx.x == g_pred_drop_cta && v == g_pred_drop_sub;
+#else
+      constexpr bool drop = false;
+#endif
+      if (lane < 4 && !drop) tma_box_2d(sbase + st * kZStage + lane * (kRowsPerCta * 128), &tm_z, full(st), c + 32 * lane, row0);
+      else if (lane >= 4 && lane < 6 && p_vec)
         tma_box_2d(sbase + kOffP + st * kPStage + (lane - 4) * 4096, &tm_p, full(st), c + 64 * (lane - 4), 0);
       if (!p_vec) {
         for (int e = lane; e < kPredLog * kSub; e += 32) {
@@ -915,5 +926,15 @@ cudaError_t launch_predictor(const PredictArgs& p, cudaStream_t stream) {
   }
   return e;
 }
+
+#ifdef DSCALE_WAIT_TEST
+// Wait-limit test build only: leave out the logit copies of sub-tile `sub` of CTA `cta` of the
+// predictor's stream kernel in every following launch; (-1, -1) switches it off.  HOST call.
+extern "C" int dscale_test_drop_pred_copy(int cta, int sub) {
+  if (cudaMemcpyToSymbol(g_pred_drop_cta, &cta, sizeof(int)) != cudaSuccess) return -3;
+  if (cudaMemcpyToSymbol(g_pred_drop_sub, &sub, sizeof(int)) != cudaSuccess) return -3;
+  return 0;
+}
+#endif
 
 }  // namespace dscale

@@ -19,7 +19,7 @@ import numpy as np
 import pytest
 import torch
 
-from dscale_inputs import CONFIGS, small_variant
+from dscale_inputs import CONFIGS, make_requests, small_variant
 from gpu_case import ALLOC_FIELDS, SCALE, attn_close, dev, full_case, oracle_attn
 
 pytestmark = pytest.mark.gpu
@@ -105,4 +105,60 @@ def test_a_wait_that_runs_out_sets_the_status_and_the_kernel_returns(wlib):
     assert status() == 0
     ok, max_abs, worst = attn_close(out, oracle_attn(req, alloc, kc, vc, qp))
     assert ok, f"second clean launch: max|d|={max_abs} at {worst}"
+    assert wlib.dscale_workspace_destroy(C.c_void_p(ws)) == 0
+
+
+def test_predictor_stream_wait_runs_out_and_the_call_returns(wlib):
+    """The same for the predictor's stream kernel: one CTA never gets the logit boxes of its second
+    sub-tile, its compute warps run into the wait limit, raise the abort flag, the copy warp waits
+    (bounded) for what is in flight, the CTA returns, the tail kernel behind it runs on whatever
+    records there are, and the call ends with DSCALE_STATUS_TIMEOUT.  After re-initialisation the
+    same call gives the product library's result again."""
+    import paper_2609_37532_b200 as P
+    from dscale_inputs import make_predictor_inputs
+    cfg = small_variant(CONFIGS["tiny"], vocab=20480, n=3, seed=83)
+    req = make_requests(cfg, n_bs=4)
+    n_bs, hq, hkv = 4, cfg.n_q_heads, cfg.n_kv_heads
+    d = {k: (v.cuda().contiguous() if torch.is_tensor(v) else v) for k, v in make_predictor_inputs(req, 64).items()}
+    n_live = dev(np.array([req["n_live"]], dtype=np.int32))
+    # the product library's answer
+    pws = P.VerifyWorkspace(n_bs, hq, hkv)
+    want = torch.zeros((n_bs, 15), dtype=torch.float32, device="cuda")
+    P.predict_scores(pws, n_live, d["draft_logits"], cfg.vocab, d["draft_hidden"], d["p_hidden"], d["p_logit"],
+                     d["w1"], d["b1"], d["w2"], d["b2"], want)
+    torch.cuda.synchronize()
+
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    nbytes = wlib.dscale_workspace_bytes(n_bs, hq, hkv, 128, sms)
+    buf = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    ws = buf.data_ptr() + (-buf.data_ptr()) % 256
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    got = torch.zeros((n_bs, 15), dtype=torch.float32, device="cuda")
+
+    def status():
+        off = wlib.dscale_ws_field(C.c_void_p(ws), n_bs, 0) - buf.data_ptr()
+        return int(buf[off:off + 4].view(torch.int32).item())
+
+    def init():
+        assert wlib.dscale_workspace_init(C.c_void_p(ws), C.c_size_t(nbytes), n_bs, hq, hkv, 128, sms, stream) == 0
+
+    def predict():
+        rc = wlib.dscale_predict_scores(
+            C.c_void_p(ws), n_bs, _vp(n_live), _vp(d["draft_logits"]), C.c_int64(d["draft_logits"].shape[2]),
+            cfg.vocab, _vp(d["draft_hidden"]), 64, _vp(d["p_hidden"]), _vp(d["p_logit"]), _vp(d["w1"]), _vp(d["b1"]),
+            _vp(d["w2"]), _vp(d["b2"]), _vp(got), C.c_void_p(None), stream)
+        assert rc == 0
+        torch.cuda.synchronize()          # returns: the kernels ended by themselves
+
+    init()
+    assert wlib.dscale_test_drop_pred_copy(0, 1) == 0
+    predict()
+    assert status() & 8, "DSCALE_STATUS_TIMEOUT was not set"
+    assert status() & ~8 == 0
+    assert wlib.dscale_test_drop_pred_copy(-1, -1) == 0
+    init()
+    got.zero_()
+    predict()
+    assert status() == 0
+    np.testing.assert_array_equal(got.cpu().numpy(), want.cpu().numpy())
     assert wlib.dscale_workspace_destroy(C.c_void_p(ws)) == 0
