@@ -31,6 +31,10 @@
 
 namespace dscale {
 
+#ifdef DSCALE_WAIT_TEST
+__device__ int g_lm_drop_cta = -1, g_lm_drop_step = -1;
+#endif
+
 namespace {
 
 constexpr int kThreads = 192;
@@ -215,7 +219,7 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
   const uint32_t bar0 = base + off_bar;
   auto bar = [&](int b) { return bar0 + 8u * b; };
   const int B_FULL = 0, B_EMPTY = sh.stages, B_ACC_FULL = 2 * sh.stages, B_ACC_EMPTY = B_ACC_FULL + 1,
-            B_GROUP = B_ACC_FULL + 2;
+            B_GROUP = B_ACC_FULL + 2, B_DRAIN = B_ACC_FULL + 3;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int c = blockIdx.x, C = gridDim.x;
@@ -227,7 +231,8 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
     mbar_init(bar(B_ACC_FULL), 1);
     mbar_init(bar(B_ACC_EMPTY), kEpiThreads);
     mbar_init(bar(B_GROUP), kEpiThreads);
-    *s_abort = 0;
+    mbar_init(bar(B_DRAIN), 1);
+    s_abort[0] = 0; s_abort[2] = 0; s_abort[3] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 5) {
@@ -257,7 +262,7 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
     const CUtensorMap* map = is_a ? &tm_a : &tm_b;
     const uint32_t dst_off = (is_a ? lane : M_TILES) * kATile;
     const uint32_t tx_bytes = M_TILES * (uint32_t)sh.a_rows * kKStep * 2 + (uint32_t)sh.n_tile * kKStep * 2;
-    int slot = 0;
+    int slot = 0, issued = 0;
     uint32_t empty_parity = 1, st = base;
     bool ok = true;
     for (int t = 0; t < my_tiles && ok; ++t) {
@@ -267,9 +272,25 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
         if (!ok) break;
         if (lane == 0) mbar_expect_tx(bar(B_FULL + slot), tx_bytes);
         __syncwarp();
-        if (is_a || is_b) tma_load_2d(st + dst_off, map, bar(B_FULL + slot), kb * kKStep, c1);
+#ifdef DSCALE_WAIT_TEST
+        // wait-limit test build only: the weight box of one k step of one CTA is left out (the
+        // barrier stays armed), so that every wait behind it runs into its limit
+        const bool drop = is_b && c == g_lm_drop_cta && issued == g_lm_drop_step;
+#else
+        constexpr bool drop = false;
+#endif
+        if ((is_a || is_b) && !drop) tma_load_2d(st + dst_off, map, bar(B_FULL + slot), kb * kKStep, c1);
+        ++issued;
         st += sh.stage_bytes;
         if (++slot == sh.stages) { slot = 0; empty_parity ^= 1; st = base; }
+      }
+    }
+    if (!ok) {
+      // a wait ran out: before shared memory is given back, wait (bounded, on a flag of its own) for
+      // the copies of the last ring's worth of k steps, each on the phase it was armed for
+      for (int back = 1; back <= sh.stages && back <= issued; ++back) {
+        const int it = issued - back;
+        mbar_wait(bar(B_FULL + it % sh.stages), (uint32_t)(it / sh.stages) & 1u, s_abort + 2);
       }
     }
     __syncwarp();
@@ -304,6 +325,11 @@ lm_head_kernel(LmArgs a, WsLayout L, LmShape sh, const __grid_constant__ CUtenso
           if (++slot == sh.stages) { slot = 0; full_parity ^= 1; st_lo = base >> 4; }
         }
         if (ok) umma_commit(bar(B_ACC_FULL));
+      }
+      if (!ok) {
+        // a wait ran out: the products issued so far must have finished before tensor memory is released
+        umma_commit(bar(B_DRAIN));
+        mbar_wait(bar(B_DRAIN), 0, s_abort + 3);
       }
     }
     __syncwarp();
@@ -426,7 +452,7 @@ lm_head_pair_kernel(LmArgs a, WsLayout L, PairShape sh, const __grid_constant__ 
   const uint32_t bar0 = base + off_bar;
   auto bar = [&](int b) { return bar0 + 8u * b; };
   const int B_FULL = 0, B_EMPTY = sh.stages, B_ACC_FULL = 2 * sh.stages, B_ACC_EMPTY = B_ACC_FULL + 1,
-            B_GROUP = B_ACC_FULL + 2;
+            B_GROUP = B_ACC_FULL + 2, B_DRAIN = B_ACC_FULL + 3;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_rank();              // 0 = leader (issues the MMAs)
@@ -439,7 +465,8 @@ lm_head_pair_kernel(LmArgs a, WsLayout L, PairShape sh, const __grid_constant__ 
     mbar_init(bar(B_ACC_FULL), 1);
     mbar_init(bar(B_ACC_EMPTY), 2 * kEpiThreads);    // the epilogue threads of both CTAs
     mbar_init(bar(B_GROUP), kEpiThreads);
-    *s_abort = 0;
+    mbar_init(bar(B_DRAIN), 1);
+    s_abort[0] = 0; s_abort[2] = 0; s_abort[3] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 5) {
@@ -474,7 +501,7 @@ lm_head_pair_kernel(LmArgs a, WsLayout L, PairShape sh, const __grid_constant__ 
     const uint32_t dst_off = is_a ? lane * kATile : M_PAIRS * kATile + j * sh.b_bytes;
     const uint32_t payload = (uint32_t)M_PAIRS * kATile + (uint32_t)N_ACC * half * kKStep * 2;
     const uint32_t full0 = map_to_cta(bar(B_FULL), 0);           // the leader's full barriers
-    int slot = 0;
+    int slot = 0, issued = 0;
     uint32_t empty_parity = 1, st = base;
     bool ok = true;
     for (int t = 0; t < my_passes && ok; ++t) {
@@ -485,8 +512,18 @@ lm_head_pair_kernel(LmArgs a, WsLayout L, PairShape sh, const __grid_constant__ 
         if (lane == 0 && rank == 0) mbar_expect_tx(bar(B_FULL + slot), 2 * payload);
         __syncwarp();
         if (is_a || is_b) tma_load_2d_pair(st + dst_off, map, full0 + 8u * slot, kb * kKStep, c1);
+        ++issued;
         st += sh.stage_bytes;
         if (++slot == sh.stages) { slot = 0; empty_parity ^= 1; st = base; }
+      }
+    }
+    if (!ok && rank == 0) {
+      // a wait ran out: the full barriers live in this CTA and count the bytes of both CTAs, so the
+      // leader waits (bounded, on a flag of its own) for the last ring's worth of k steps it armed;
+      // the peer stays in the cluster barrier at the end until the leader is through
+      for (int back = 1; back <= sh.stages && back <= issued; ++back) {
+        const int it = issued - back;
+        mbar_wait(bar(B_FULL + it % sh.stages), (uint32_t)(it / sh.stages) & 1u, s_abort + 2);
       }
     }
     __syncwarp();
@@ -529,6 +566,12 @@ lm_head_pair_kernel(LmArgs a, WsLayout L, PairShape sh, const __grid_constant__ 
           umma_commit_pair(bar(B_ACC_FULL));
           umma_commit_pair(peer_bar0 + 8u * B_ACC_FULL);
         }
+      }
+      if (!ok) {
+        // a wait ran out: the products issued so far (they write both CTAs' tensor memory) must have
+        // finished before either CTA releases it; both stay in the cluster barrier until then
+        umma_commit_pair(bar(B_DRAIN));
+        mbar_wait(bar(B_DRAIN), 0, s_abort + 3);
       }
     }
     __syncwarp();
@@ -713,5 +756,16 @@ cudaError_t launch_lm_head(void* ws, int n_bs, const void* hidden, const void* w
   lm_head_kernel<1><<<num_ctas, kThreads, sh.smem_bytes, stream>>>(a, L, sh, ta, tb);
   return cudaGetLastError();
 }
+
+#ifdef DSCALE_WAIT_TEST
+// Wait-limit test build only: leave out the weight copy of k step `step` (counted from the CTA's
+// first) of CTA `cta` of the one-CTA-per-tile LM-head kernel in every following launch; (-1, -1)
+// switches it off.  HOST call.
+extern "C" int dscale_test_drop_lm_copy(int cta, int step) {
+  if (cudaMemcpyToSymbol(g_lm_drop_cta, &cta, sizeof(int)) != cudaSuccess) return -3;
+  if (cudaMemcpyToSymbol(g_lm_drop_step, &step, sizeof(int)) != cudaSuccess) return -3;
+  return 0;
+}
+#endif
 
 }  // namespace dscale

@@ -162,3 +162,73 @@ def test_predictor_stream_wait_runs_out_and_the_call_returns(wlib):
     assert status() == 0
     np.testing.assert_array_equal(got.cpu().numpy(), want.cpu().numpy())
     assert wlib.dscale_workspace_destroy(C.c_void_p(ws)) == 0
+
+
+def test_lm_head_wait_runs_out_and_the_call_returns(wlib):
+    """The same for the one-CTA-per-tile LM-head kernel: one CTA never gets the weight box of its
+    second k step; its MMA warp runs into the wait limit, waits (bounded) for the products it has
+    issued, the copy warp waits (bounded) for the copies it has armed, the epilogue warps leave,
+    tensor memory is released and the kernel returns with DSCALE_STATUS_TIMEOUT.  After
+    re-initialisation the same call gives the product library's outputs."""
+    import paper_2609_37532_b200 as P
+    from dscale_inputs import make_lm_head_unpacked, rows_to_packed
+    from gpu_case import StagedRequests, gpu_alloc, oracle_alloc
+    cfg = small_variant(CONFIGS["tiny"], vocab=20000, n=7, seed=85)
+    req = make_requests(cfg, n_bs=8)
+    n_bs, n, hq, hkv, H = 8, req["n_live"], cfg.n_q_heads, cfg.n_kv_heads, 512
+    alloc = oracle_alloc(req)
+    weight, hid_unpacked = make_lm_head_unpacked(req, H)
+    hidden = rows_to_packed(hid_unpacked, alloc["k"], alloc["offset"], n, 8 * n_bs).cuda().contiguous()
+    weight = weight.cuda().contiguous()
+
+    def outputs():
+        return [torch.full((n_bs,), -9, dtype=torch.int32, device="cuda"),
+                torch.full((n_bs,), -9, dtype=torch.int32, device="cuda"),
+                torch.full((n_bs, 16), -9, dtype=torch.int32, device="cuda"),
+                torch.full((n_bs,), -9, dtype=torch.int32, device="cuda")]
+
+    # the product library's answer
+    pws = P.VerifyWorkspace(n_bs, hq, hkv)
+    gpu_alloc(P, pws, StagedRequests(req))
+    want = outputs()
+    P.lm_head_accept(pws, hidden, weight, want[0], want[1], want[2], want[3])
+    torch.cuda.synchronize()
+    assert pws.status() == 0
+
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    nbytes = wlib.dscale_workspace_bytes(n_bs, hq, hkv, 128, sms)
+    buf = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    ws = buf.data_ptr() + (-buf.data_ptr()) % 256
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    n_live = dev(np.array([n], dtype=np.int32))
+    scores, draft = dev(req["scores"]), dev(req["draft_tokens"])
+    ctx, bt = dev(req["ctx_len"]), dev(req["block_table"])
+
+    def status():
+        off = wlib.dscale_ws_field(C.c_void_p(ws), n_bs, 0) - buf.data_ptr()
+        return int(buf[off:off + 4].view(torch.int32).item())
+
+    def init_and_alloc():
+        assert wlib.dscale_workspace_init(C.c_void_p(ws), C.c_size_t(nbytes), n_bs, hq, hkv, 128, sms, stream) == 0
+        assert wlib.dscale_alloc_verify(C.c_void_p(ws), n_bs, _vp(n_live), _vp(scores), 0, _vp(draft), _vp(ctx),
+                                        _vp(bt), req["max_pages"], req["num_pages"], stream) == 0
+
+    def lm_head(o):
+        rc = wlib.dscale_lm_head_accept(C.c_void_p(ws), n_bs, _vp(hidden), _vp(weight), H, cfg.vocab, _vp(o[0]),
+                                        _vp(o[1]), _vp(o[2]), _vp(o[3]), C.c_void_p(None), C.c_void_p(None), stream)
+        assert rc == 0
+        torch.cuda.synchronize()          # returns: the kernel ended by itself
+
+    init_and_alloc()
+    assert wlib.dscale_test_drop_lm_copy(0, 1) == 0
+    lm_head(outputs())
+    assert status() & 8, "DSCALE_STATUS_TIMEOUT was not set"
+    assert status() & ~8 == 0
+    assert wlib.dscale_test_drop_lm_copy(-1, -1) == 0
+    init_and_alloc()
+    got = outputs()
+    lm_head(got)
+    assert status() == 0
+    for g, w in zip(got, want):
+        np.testing.assert_array_equal(g.cpu().numpy(), w.cpu().numpy())
+    assert wlib.dscale_workspace_destroy(C.c_void_p(ws)) == 0
